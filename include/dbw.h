@@ -1,0 +1,191 @@
+/*
+ * dbw.h — C ABI of the cb-DyBW round library (consensus SGD with dynamic backup workers,
+ * arXiv 2102.06280) for one NVIDIA B200.
+ *
+ * N workers are simulated together.  Row i of the row-major N x ld fp32 matrix X is worker
+ * i's parameter vector w_i (the paper stores workers as columns of W; this is its transpose).
+ * The communication graph is undirected, connected, without self loops, and is given once as
+ * sorted CSR (rowptr[N+1], col[nnz]); deg_i = rowptr[i+1] - rowptr[i].  b_i is the number of
+ * backup workers of i and p_i = deg_i - b_i the number of neighbours it waits for.
+ *
+ * Conventions for every entry point
+ *   - returns DBW_OK (0) or a negative DBW_ERR_* detected on the host before anything is
+ *     launched; nothing is printed.
+ *   - pointers marked DEVICE are device memory owned by the caller (never freed, reallocated
+ *     or retained past the call unless stated); pointers marked HOST are host memory.
+ *   - all device work is enqueued on the `stream` argument (a cudaStream_t passed as void*)
+ *     and is asynchronous; the caller synchronises.
+ *   - conditions that only the device can see (b_i outside [0, deg_i], NaN arrival time,
+ *     a pipeline wait that ran out) set bits in a status word read by dbw_status(); the
+ *     kernels clamp and continue, they never trap.
+ */
+#ifndef DBW_H
+#define DBW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dbw_handle dbw_handle;
+
+enum {
+    DBW_OK = 0,
+    DBW_ERR_NULL = -1,       /* a required pointer is NULL */
+    DBW_ERR_BAD_GRAPH = -2,  /* CSR unsorted, asymmetric, self loop, index out of range, disconnected */
+    DBW_ERR_BAD_SHAPE = -3,  /* N < 1, ld < d, ld % 4 != 0, pointer not 16-byte aligned, illegal aliasing */
+    DBW_ERR_BAD_B = -4,      /* host-side b outside [0, deg] */
+    DBW_ERR_BAD_MODEL = -5,  /* model descriptor inconsistent with d / ld, or no model / data set */
+    DBW_ERR_CUDA = -6,       /* a CUDA runtime call failed; see dbw_last_cuda_error() */
+    DBW_ERR_STATE = -7       /* state blob of the wrong size or version */
+};
+
+/* flags of dbw_init */
+#define DBW_WEIGHT_METROPOLIS 0u /* Assumption 1: w_ij = 1/(1+max{p_i,p_j}), w_ii = 1 - sum */
+#define DBW_WEIGHT_UNIFORM 1u    /* w_ii = w_ij = 1/(1+p_i) over self and the kept neighbours */
+#define DBW_ORDER_LOCAL_THEN_MIX 0u   /* Algorithm 1, Eqs. 4-5 */
+#define DBW_ORDER_MIX_THEN_CORRECT 2u /* Eq. 3 restricted to the kept set */
+#define DBW_GEMM_FP32 0u /* dense layers in fp32 on the CUDA cores */
+#define DBW_GEMM_BF16 4u /* dense layers with BF16 operands on tcgen05 tensor cores, fp32 accumulate */
+
+/* bits of the device status word */
+#define DBW_STATUS_BAD_B 1u       /* some b_i was outside [0, deg_i] (clamped) */
+#define DBW_STATUS_NAN_TIME 2u    /* some arrival time was NaN (ordered last) */
+#define DBW_STATUS_WAIT_TIMEOUT 4u /* a bounded pipeline wait expired; results of that call are invalid */
+#define DBW_STATUS_BAD_INDEX 8u   /* a batch index was outside [0, S) (clamped) */
+
+#define DBW_MAX_LAYERS 8
+
+/*
+ * Model: ReLU MLP dims[0] -> dims[1] -> ... -> dims[n_layers] with mean softmax cross-entropy
+ * (Eq. 2: the mini-batch stochastic gradient g(w_j)).  Layer l (0-based) has W_l stored
+ * row-major [dims[l+1]][dims[l]] at float offset w_off[l] of a parameter row and its bias at
+ * b_off[l].  Offsets are multiples of 32 floats; the gaps and the tail up to ld are padding
+ * that stays zero.  dbw_model_layout() fills a descriptor with the canonical padded layout.
+ */
+typedef struct {
+    int32_t n_layers;
+    int32_t dims[DBW_MAX_LAYERS + 1];
+    int64_t w_off[DBW_MAX_LAYERS];
+    int64_t b_off[DBW_MAX_LAYERS];
+    int32_t batch; /* mini-batch size |C_j(k)| per worker */
+} dbw_model_desc;
+
+/* Canonical padded layout.  HOST in: dims[n_layers+1], batch; out: *desc, *d (logical
+ * parameter count: sum of out*in + out), *ld (padded row length, multiple of 32). */
+int dbw_model_layout(const int32_t* dims, int32_t n_layers, int32_t batch, dbw_model_desc* desc,
+                     int64_t* d, int64_t* ld);
+
+/*
+ * Section 2.1 (graph, neighbourhoods) and Algorithm 2's input (the link set P).
+ * Validates and copies the HOST CSR, builds P as the breadth-first spanning tree from worker 0
+ * (neighbours in ascending index, links in discovery order), allocates the workspace on
+ * `device` and returns the handle.  `model` may be NULL (mixing only: gradients are supplied
+ * to dbw_round / dbw_mix).  The handle owns only its workspace.
+ */
+int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* h_rowptr,
+             const int32_t* h_col, const dbw_model_desc* model, uint32_t flags, int device);
+int dbw_destroy(dbw_handle* h);
+
+/* Local data sets D_j (Section 2.1).  DEVICE feat [N][S][dims[0]] fp32, labels [N][S] int32 in
+ * [0, dims[L]).  The pointers are retained (not copied) until replaced or the handle dies. */
+int dbw_set_dataset(dbw_handle* h, const float* feat, const int32_t* labels, int32_t S);
+
+/*
+ * Section 2.2 (worker j waits for the first p_j updates) and Section 3.2.2 (T_j, T).
+ * DEVICE in : t[N] f64 arrival time of each worker's update, b[N] int32.
+ * DEVICE out: kept[nnz] uint8 aligned with col (1 = waited for, 0 = backup); ties in t go to
+ *             the lower worker index;
+ *             T_nbr[N]    max t over the kept neighbours (0.0 when p_i = 0);
+ *             T_worker[N] max(t_i, T_nbr[i]) when p_i >= 1; t_i when i is only waited for by
+ *                         others; 0.0 when i takes no part;
+ *             T_round[1]  max t over the workers that take part (0.0 if none).
+ * Only comparisons are applied to t, so the outputs are bit-exact.  Any out pointer but kept
+ * may be NULL.
+ */
+int dbw_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kept, double* T_worker,
+               double* T_nbr, double* T_round, void* stream);
+
+/*
+ * Eq. 2.  DEVICE in: X [N][ld]; batch_idx [N][batch] int32 sample indices into the data set.
+ * DEVICE out: G [N][ld] fp32, g(w_i) in the layout of X (padding untouched: pass it zeroed);
+ * loss [N] fp32 mean cross-entropy of each worker's batch (nullable).
+ */
+int dbw_grad(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss,
+             void* stream);
+
+/*
+ * Assumption 1 (weights) + Eqs. 4-5 or Eq. 3 (update), every row read from the OLD X.
+ * DEVICE in : X [N][ld], G [N][ld], kept[nnz], b[N]; lr scalar; lr_per_worker[N] fp32 nullable
+ *             (eta_j; overrides lr).
+ * DEVICE out: X_out [N][ld].  X_out may alias X exactly (in place) when dbw_mix_in_place_ok()
+ *             is 1; partial overlap is an error.  G is read only.
+ * Summation order per element is fixed (self, then kept neighbours in CSR order), so results
+ * are reproducible run to run.
+ */
+int dbw_mix(dbw_handle* h, const float* X, const float* G, const uint8_t* kept, const int32_t* b,
+            float lr, const float* lr_per_worker, float* X_out, void* stream);
+int dbw_mix_in_place_ok(const dbw_handle* h);
+/* Expert knob: columns per shared-memory panel of the mix kernel: 0 = automatic, 16 / 32 / 64 /
+ * 128 = fixed (falls back to the direct kernel when N * cols * 4 bytes exceed shared memory),
+ * -1 = always the direct (L2 re-read, out-of-place only) kernel. */
+int dbw_set_mix_panel(dbw_handle* h, int32_t cols);
+
+/*
+ * Algorithm 1, one iteration: gradients (dbw_grad, or G_ext when batch_idx is NULL), selection
+ * (dbw_select) and the update (dbw_mix) in one call.  Arguments as in those three; loss is
+ * nullable; G_ext [N][ld] is used iff batch_idx == NULL.
+ */
+int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
+              const int32_t* batch_idx, const float* G_ext, float lr, const float* lr_per_worker,
+              float* X_out, uint8_t* kept, double* T_worker, double* T_nbr, double* T_round,
+              float* loss, void* stream);
+
+/*
+ * The same round for callers whose per-round inputs live in HOST memory (pinned memory makes
+ * the copies asynchronous).  X / X_out / G_ext stay DEVICE (the parameters are the state of the
+ * simulation); h_t[N], h_b[N], h_batch_idx[N][batch] are copied to the device on `stream`, the
+ * round runs, and h_kept[nnz], h_T_worker[N], h_T_round[1], h_loss[N] (each nullable) are copied
+ * back on `stream`.  The call does not synchronise.
+ */
+int dbw_round_host(dbw_handle* h, const float* X, const double* h_t, const int32_t* h_b,
+                   const int32_t* h_batch_idx, const float* G_ext, float lr, float* X_out,
+                   uint8_t* h_kept, double* h_T_worker, double* h_T_round, float* h_loss,
+                   void* stream);
+
+/*
+ * Section 4.1 (threshold rule) and Algorithm 2 (one iteration of the epoch).
+ * DEVICE in : t_next[N] f64, the arrival times of the round about to run.
+ * DEVICE out: b_out[N] int32, theta_out[1] f64 (nullable).
+ * theta = the smallest max(t_u, t_v) over the links (u,v) of P not yet covered in this epoch
+ * (first such link on ties); that link becomes covered; after |P| = N-1 calls the covered set
+ * is emptied.  Then p_j = #{i in N_j : t_i <= theta} if t_j <= theta, else 0; b_j = deg_j - p_j.
+ * The epoch state lives on the device and advances in stream order.
+ */
+int dbw_update_backups(dbw_handle* h, const double* t_next, int32_t* b_out, double* theta_out,
+                       void* stream);
+int dbw_reset_backups(dbw_handle* h, void* stream); /* empty the covered set, restart the epoch */
+
+/* Epoch state (covered links, position in the epoch) as an opaque blob, for resuming a run.
+ * HOST buf; *size in: capacity, out: bytes needed/written.  Both synchronise `stream`. */
+int dbw_state_export(dbw_handle* h, void* buf, size_t* size, void* stream);
+int dbw_state_import(dbw_handle* h, const void* buf, size_t size, void* stream);
+
+/* Device status word (DBW_STATUS_* bits, accumulated since the last call); synchronises the
+ * device.  Returns the bits (>= 0) or a negative error. */
+int dbw_status(dbw_handle* h);
+
+/* Spanning links P on the HOST: links[2*(N-1)] receives (u,v) pairs; returns N-1 or an error. */
+int dbw_get_links(const dbw_handle* h, int32_t* links);
+
+/* Kernels launched by this library since it was loaded (for launch accounting). */
+int64_t dbw_launch_count(void);
+/* cudaError_t of the last failing runtime call in this library (0 if none). */
+int dbw_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBW_H */

@@ -1,0 +1,128 @@
+// Shared declarations of the cb-DyBW round library: the handle and the host-side launchers
+// each translation unit provides.  No device code crosses translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "dbw.h"
+
+namespace dbw {
+
+extern std::atomic<long long> g_launches;
+extern std::atomic<int> g_last_cuda_error;
+
+inline bool cuda_ok(cudaError_t e) {
+    if (e != cudaSuccess) {
+        g_last_cuda_error.store((int)e);
+        return false;
+    }
+    return true;
+}
+
+#define DBW_CUDA(call)                                  \
+    do {                                                \
+        if (!::dbw::cuda_ok((call))) return DBW_ERR_CUDA; \
+    } while (0)
+
+// Counts a kernel launch and reports a launch-configuration failure.
+#define DBW_LAUNCHED()                                         \
+    do {                                                       \
+        ::dbw::g_launches.fetch_add(1);                        \
+        if (!::dbw::cuda_ok(cudaGetLastError())) return DBW_ERR_CUDA; \
+    } while (0)
+
+// Per-round mixing plan (built on the device from kept and b): for each worker the compacted
+// list of kept neighbours with their weights, padded to `stride` entries with (self, 0).
+struct MixPlan {
+    int* idx = nullptr;      // [N][stride]
+    float* w = nullptr;      // [N][stride]
+    float* w_self = nullptr; // [N]
+    int* cnt = nullptr;      // [N]
+    int stride = 0;
+};
+
+struct BF16State;  // tensor-core gradient path (grad_bf16.cu)
+
+}  // namespace dbw
+
+struct dbw_handle {
+    int N = 0;
+    int64_t d = 0, ld = 0;
+    int nnz = 0;
+    int maxdeg = 0;
+    uint32_t flags = 0;
+    int device = 0;
+    int sm_count = 0;
+    int smem_optin = 0;  // max dynamic shared memory per block
+
+    std::vector<int32_t> h_rowptr, h_col, h_links;  // host copies; links = (u,v) pairs of P
+    int32_t* d_rowptr = nullptr;
+    int32_t* d_col = nullptr;
+    int32_t* d_links = nullptr;  // [2*(N-1)]
+
+    // Algorithm 2 state, device resident: covered[N-1] flags then step counter
+    int32_t* d_covered = nullptr;  // [N-1]
+    int32_t* d_epoch = nullptr;    // [2]: links covered in this epoch, position of last credited link
+
+    uint32_t* d_status = nullptr;    // [1]
+    uint32_t* d_waited = nullptr;    // [N] scratch flags of the selection kernel (kept zero between calls)
+    uint32_t* d_ticket = nullptr;    // [1] block ticket of the selection kernel (kept zero between calls)
+    double* d_Tnbr_ws = nullptr;     // [N]
+
+    dbw::MixPlan plan;
+    int mix_panel_cols = 0;  // 0 = automatic
+
+    // model / gradient path
+    bool has_model = false;
+    dbw_model_desc model{};
+    const float* feat = nullptr;
+    const int32_t* labels = nullptr;
+    int32_t S = 0;
+    float* d_act[DBW_MAX_LAYERS + 1] = {};  // fp32 path: A_0 (gathered batch) .. A_L (logits), [N][B][dims[l]]
+    float* d_dz[DBW_MAX_LAYERS + 1] = {};   // fp32 path: dZ_l for l = 1..L, [N][B][dims[l]]
+    int32_t* d_ylab = nullptr;              // [N][B] gathered labels
+    float* d_G = nullptr;                   // [N][ld] gradient workspace of dbw_round (lazy)
+    dbw::BF16State* bf16 = nullptr;
+
+    // device staging of dbw_round_host
+    double* s_t = nullptr;
+    int32_t* s_b = nullptr;
+    int32_t* s_bidx = nullptr;
+    uint8_t* s_kept = nullptr;
+    double* s_Tw = nullptr;
+    double* s_Tr = nullptr;
+    float* s_loss = nullptr;
+};
+
+namespace dbw {
+
+// select.cu
+int launch_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kept, double* T_worker,
+                  double* T_nbr, double* T_round, bool build_plan, cudaStream_t s);
+int launch_plan_from_kept(dbw_handle* h, const uint8_t* kept, const int32_t* b, cudaStream_t s);
+
+// mix.cu
+int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+               cudaStream_t s);
+bool mix_panel_fits(const dbw_handle* h);
+
+// dtur.cu
+int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);
+
+// grad_fp32.cu
+int grad_fp32_alloc(dbw_handle* h);
+void grad_fp32_free(dbw_handle* h);
+int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss,
+                     cudaStream_t s);
+
+// grad_bf16.cu
+int grad_bf16_alloc(dbw_handle* h);
+void grad_bf16_free(dbw_handle* h);
+int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss,
+                     cudaStream_t s);
+
+}  // namespace dbw

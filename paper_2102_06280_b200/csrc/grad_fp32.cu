@@ -1,0 +1,235 @@
+// Mini-batch stochastic gradient (Eq. 2) of the ReLU MLP with softmax cross-entropy, fp32 on the
+// CUDA cores, for all workers at once: every kernel is batched over workers (blockIdx.z), whose
+// weights are slices of their rows of X.
+#include "common.cuh"
+
+namespace dbw {
+
+namespace {
+
+// ------------------------------------------------------------------ batch gather
+__global__ void gather_batch_kernel(int B, int S, int in_dim, const float* __restrict__ feat,
+                                    const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
+                                    float* __restrict__ A0, int32_t* __restrict__ ylab, uint32_t* status) {
+    const int s = blockIdx.x, i = blockIdx.y;
+    int src = batch_idx[(size_t)i * B + s];
+    if (src < 0 || src >= S) {
+        if (threadIdx.x == 0) atomicOr(status, DBW_STATUS_BAD_INDEX);
+        src = src < 0 ? 0 : S - 1;
+    }
+    const float* from = feat + ((size_t)i * S + src) * in_dim;
+    float* to = A0 + ((size_t)i * B + s) * in_dim;
+    if ((in_dim & 3) == 0) {
+        for (int k = threadIdx.x; k < in_dim / 4; k += blockDim.x)
+            reinterpret_cast<float4*>(to)[k] = __ldg(reinterpret_cast<const float4*>(from) + k);
+    } else {
+        for (int k = threadIdx.x; k < in_dim; k += blockDim.x) to[k] = from[k];
+    }
+    if (threadIdx.x == 0) ylab[(size_t)i * B + s] = labels[(size_t)i * S + src];
+}
+
+// ------------------------------------------------------------------ batched strided GEMM
+// C[z][m][n] = epilogue( sum_k A[z](m,k) * B[z](k,n) ), operands addressed through strides so
+// that the same kernel serves Z = A W^T, dW = dZ^T A and dA = dZ W.
+struct GemmArgs {
+    const float* A;
+    long long sAz, sAm, sAk;
+    const float* B;
+    long long sBz, sBn, sBk;
+    float* C;
+    long long sCz, sCm;
+    const float* bias;  // indexed by n, nullable
+    long long sBiasz;
+    const float* mask;  // same shape as C, nullable: C *= (mask > 0)
+    long long sMz, sMm;
+    int M, N, K;
+    int relu;
+};
+
+constexpr int TM = 64, TN = 64, TK = 16;
+
+__global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
+    __shared__ __align__(16) float As[TK][TM + 4];
+    __shared__ __align__(16) float Bs[TK][TN + 4];
+    const int z = blockIdx.z;
+    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+    const float* A = g.A + (size_t)z * g.sAz;
+    const float* B = g.B + (size_t)z * g.sBz;
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const bool a_k_fast = g.sAk == 1;
+    const bool b_k_fast = g.sBk == 1;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < g.K; k0 += TK) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int e = tid + r * 256;
+            const int ka = a_k_fast ? (e & 15) : (e >> 6);
+            const int ma = a_k_fast ? (e >> 4) : (e & 63);
+            float v = 0.f;
+            if (m0 + ma < g.M && k0 + ka < g.K) v = __ldg(A + (size_t)(m0 + ma) * g.sAm + (size_t)(k0 + ka) * g.sAk);
+            As[ka][ma] = v;
+            const int kb = b_k_fast ? (e & 15) : (e >> 6);
+            const int nb = b_k_fast ? (e >> 4) : (e & 63);
+            v = 0.f;
+            if (n0 + nb < g.N && k0 + kb < g.K) v = __ldg(B + (size_t)(n0 + nb) * g.sBn + (size_t)(k0 + kb) * g.sBk);
+            Bs[kb][nb] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < TK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+            const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float* C = g.C + (size_t)z * g.sCz;
+    const float* bias = g.bias ? g.bias + (size_t)z * g.sBiasz : nullptr;
+    const float* mask = g.mask ? g.mask + (size_t)z * g.sMz : nullptr;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= g.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= g.N) continue;
+            float v = acc[i][j];
+            if (bias) v += bias[n];
+            if (g.relu) v = fmaxf(v, 0.f);
+            if (mask && !(mask[(size_t)m * g.sMm + n] > 0.f)) v = 0.f;
+            C[(size_t)m * g.sCm + n] = v;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ softmax cross-entropy
+// One CTA per worker, one warp per sample at a time.  dZ = (softmax(z) - onehot(y)) / B;
+// loss = mean over the batch of (logsumexp(z) - z_y), summed in a fixed order.
+__global__ void __launch_bounds__(256)
+softmax_ce_kernel(int B, int C, const float* __restrict__ logits, const int32_t* __restrict__ ylab,
+                  float* __restrict__ dz, float* __restrict__ loss) {
+    const int i = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float invB = 1.0f / (float)B;
+    float wloss = 0.f;
+    for (int s = warp; s < B; s += 8) {
+        const float* z = logits + ((size_t)i * B + s) * C;
+        float* o = dz + ((size_t)i * B + s) * C;
+        const int y = ylab[(size_t)i * B + s];
+        float mx = -INFINITY;
+        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+#pragma unroll
+        for (int k = 16; k > 0; k >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, k));
+        float sum = 0.f;
+        for (int c = lane; c < C; c += 32) sum += expf(z[c] - mx);
+#pragma unroll
+        for (int k = 16; k > 0; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+        const float inv = 1.0f / sum;
+        for (int c = lane; c < C; c += 32) o[c] = (expf(z[c] - mx) * inv - (c == y ? 1.f : 0.f)) * invB;
+        wloss += (mx + logf(sum)) - z[y];
+    }
+    __shared__ float sl[8];
+    if (lane == 0) sl[warp] = wloss;
+    __syncthreads();
+    if (threadIdx.x == 0 && loss) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += sl[w];
+        loss[i] = t * invB;
+    }
+}
+
+// db[z][o] = sum_m dZ[z][m][o]
+__global__ void bias_grad_kernel(int B, int out_dim, const float* __restrict__ dz, float* __restrict__ G,
+                                 long long ld, long long b_off) {
+    const int i = blockIdx.y;
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= out_dim) return;
+    const float* p = dz + (size_t)i * B * out_dim + o;
+    float s = 0.f;
+    for (int m = 0; m < B; ++m) s += p[(size_t)m * out_dim];
+    G[(size_t)i * ld + b_off + o] = s;
+}
+
+int run_gemm(const GemmArgs& g, int batch, cudaStream_t s) {
+    dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, batch);
+    gemm_simt_kernel<<<grid, 256, 0, s>>>(g);
+    DBW_LAUNCHED();
+    return DBW_OK;
+}
+
+}  // namespace
+
+int grad_fp32_alloc(dbw_handle* h) {
+    const dbw_model_desc& m = h->model;
+    const size_t NB = (size_t)h->N * m.batch;
+    for (int l = 0; l <= m.n_layers; ++l) {
+        DBW_CUDA(cudaMalloc(&h->d_act[l], NB * m.dims[l] * sizeof(float)));
+        if (l >= 1) DBW_CUDA(cudaMalloc(&h->d_dz[l], NB * m.dims[l] * sizeof(float)));
+    }
+    DBW_CUDA(cudaMalloc(&h->d_ylab, NB * sizeof(int32_t)));
+    return DBW_OK;
+}
+
+void grad_fp32_free(dbw_handle* h) {
+    for (int l = 0; l <= DBW_MAX_LAYERS; ++l) {
+        if (h->d_act[l]) cudaFree(h->d_act[l]);
+        if (h->d_dz[l]) cudaFree(h->d_dz[l]);
+        h->d_act[l] = h->d_dz[l] = nullptr;
+    }
+    if (h->d_ylab) cudaFree(h->d_ylab);
+    h->d_ylab = nullptr;
+}
+
+int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss,
+                     cudaStream_t s) {
+    const dbw_model_desc& m = h->model;
+    const int B = m.batch, L = m.n_layers, N = h->N;
+    gather_batch_kernel<<<dim3(B, N), 128, 0, s>>>(B, h->S, m.dims[0], h->feat, h->labels, batch_idx,
+                                                   h->d_act[0], h->d_ylab, h->d_status);
+    DBW_LAUNCHED();
+    int rc;
+    // forward: Z_l = A_{l-1} W_l^T + b_l, A_l = ReLU(Z_l), logits for the last layer
+    for (int l = 0; l < L; ++l) {
+        const int in = m.dims[l], out = m.dims[l + 1];
+        GemmArgs g{};
+        g.A = h->d_act[l]; g.sAz = (long long)B * in; g.sAm = in; g.sAk = 1;
+        g.B = X + m.w_off[l]; g.sBz = h->ld; g.sBn = in; g.sBk = 1;
+        g.C = h->d_act[l + 1]; g.sCz = (long long)B * out; g.sCm = out;
+        g.bias = X + m.b_off[l]; g.sBiasz = h->ld;
+        g.M = B; g.N = out; g.K = in; g.relu = l < L - 1;
+        if ((rc = run_gemm(g, N, s)) != DBW_OK) return rc;
+    }
+    softmax_ce_kernel<<<N, 256, 0, s>>>(B, m.dims[L], h->d_act[L], h->d_ylab, h->d_dz[L], loss);
+    DBW_LAUNCHED();
+    // backward
+    for (int l = L - 1; l >= 0; --l) {
+        const int in = m.dims[l], out = m.dims[l + 1];
+        GemmArgs g{};  // dW_l[o][k] = sum_m dZ[m][o] A_{l}[m][k]
+        g.A = h->d_dz[l + 1]; g.sAz = (long long)B * out; g.sAm = 1; g.sAk = out;
+        g.B = h->d_act[l]; g.sBz = (long long)B * in; g.sBn = 1; g.sBk = in;
+        g.C = G + m.w_off[l]; g.sCz = h->ld; g.sCm = in;
+        g.M = out; g.N = in; g.K = B;
+        if ((rc = run_gemm(g, N, s)) != DBW_OK) return rc;
+        bias_grad_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(B, out, h->d_dz[l + 1], G, h->ld, m.b_off[l]);
+        DBW_LAUNCHED();
+        if (l > 0) {  // dZ_{l}[m][k] = (sum_o dZ_{l+1}[m][o] W_l[o][k]) * [A_l[m][k] > 0]
+            GemmArgs a{};
+            a.A = h->d_dz[l + 1]; a.sAz = (long long)B * out; a.sAm = out; a.sAk = 1;
+            a.B = X + m.w_off[l]; a.sBz = h->ld; a.sBn = 1; a.sBk = in;
+            a.C = h->d_dz[l]; a.sCz = (long long)B * in; a.sCm = in;
+            a.mask = h->d_act[l]; a.sMz = (long long)B * in; a.sMm = in;
+            a.M = B; a.N = in; a.K = out;
+            if ((rc = run_gemm(a, N, s)) != DBW_OK) return rc;
+        }
+    }
+    return DBW_OK;
+}
+
+}  // namespace dbw

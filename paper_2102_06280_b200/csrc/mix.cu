@@ -1,0 +1,173 @@
+// Masked consensus mix fused with the SGD step (Eqs. 4-5, or Eq. 3 over the kept set).
+//
+// Panel kernel: a CTA owns a panel of `4*GS` consecutive columns of ALL N rows.  It streams the
+// panel of X and G from HBM once (128-bit loads), forms the locally updated rows x - lr*g on
+// the fly and parks them in shared memory; then every output row of the panel is a weighted sum
+// of shared-memory rows, written once with 128-bit stores.  Each element of X and G is read from
+// HBM once and each element of X' is written once (12 bytes per parameter element).  A panel is
+// fully staged before any of it is written and panels are disjoint, so X' may overwrite X.
+#include "common.cuh"
+
+namespace dbw {
+
+namespace {
+
+constexpr int kMixThreads = 512;
+
+__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+
+__device__ __forceinline__ float4 fma4(float w, float4 v, float4 a) {
+    a.x = fmaf(w, v.x, a.x);
+    a.y = fmaf(w, v.y, a.y);
+    a.z = fmaf(w, v.z, a.z);
+    a.w = fmaf(w, v.w, a.w);
+    return a;
+}
+
+template <int GS>
+__global__ void __launch_bounds__(kMixThreads)
+mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ G, float lr,
+                 const float* __restrict__ lr_pw, float* Xout, MixPlan plan, int mix_then_correct,
+                 int n_panels) {
+    extern __shared__ float4 sm[];  // [N][GS]
+    const int tid = threadIdx.x;
+    const int q = tid % GS;
+    const int gid = tid / GS;
+    constexpr int kGroups = kMixThreads / GS;
+    const int total = N * GS;
+
+    for (int panel = blockIdx.x; panel < n_panels; panel += gridDim.x) {
+        const long long col0 = (long long)panel * (4 * GS);
+        // ---- stage the panel: x (Eq. 3 order) or x - lr*g (Eq. 4) ----
+#pragma unroll 4
+        for (int idx = tid; idx < total; idx += kMixThreads) {
+            const int r = idx / GS;
+            const long long c = col0 + 4 * (idx % GS);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < ld) {
+                v = ldg4(X + (size_t)r * ld + c);
+                if (!mix_then_correct) {
+                    const float4 g = ldg4(G + (size_t)r * ld + c);
+                    const float nlr = -(lr_pw ? lr_pw[r] : lr);
+                    v = fma4(nlr, g, v);
+                }
+            }
+            sm[idx] = v;
+        }
+        __syncthreads();
+        // ---- every output row of the panel ----
+        const long long c = col0 + 4 * q;
+        for (int i = gid; i < N; i += kGroups) {
+            const float ws = plan.w_self[i];
+            const float4 self = sm[i * GS + q];
+            float4 acc = make_float4(ws * self.x, ws * self.y, ws * self.z, ws * self.w);
+            const int cnt = plan.cnt[i];
+            const int4* pi = reinterpret_cast<const int4*>(plan.idx + (size_t)i * plan.stride);
+            const float4* pw = reinterpret_cast<const float4*>(plan.w + (size_t)i * plan.stride);
+            for (int k = 0; k < cnt; k += 4) {
+                const int4 j = __ldg(pi + (k >> 2));
+                const float4 w = __ldg(pw + (k >> 2));
+                acc = fma4(w.x, sm[j.x * GS + q], acc);
+                acc = fma4(w.y, sm[j.y * GS + q], acc);
+                acc = fma4(w.z, sm[j.z * GS + q], acc);
+                acc = fma4(w.w, sm[j.w * GS + q], acc);
+            }
+            if (c < ld) {
+                if (mix_then_correct) {
+                    const float4 g = ldg4(G + (size_t)i * ld + c);
+                    acc = fma4(-(lr_pw ? lr_pw[i] : lr), g, acc);
+                }
+                *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Fallback for graphs too large for a shared-memory panel: one thread per 4 output columns,
+// neighbour rows re-read through L2.  Out of place only.
+__global__ void __launch_bounds__(256)
+mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float* __restrict__ G, float lr,
+                  const float* __restrict__ lr_pw, float* __restrict__ Xout, MixPlan plan,
+                  int mix_then_correct) {
+    const long long ld4 = ld / 4;
+    const long long total = (long long)N * ld4;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        // consecutive threads walk down the rows of one column group so that neighbour reads of
+        // concurrently running threads fall in the same few columns (L2 reuse)
+        const int i = (int)(e % N);
+        const long long c = 4 * (e / N);
+        auto stepped = [&](int r) {
+            float4 v = ldg4(X + (size_t)r * ld + c);
+            if (!mix_then_correct) v = fma4(-(lr_pw ? lr_pw[r] : lr), ldg4(G + (size_t)r * ld + c), v);
+            return v;
+        };
+        const float ws = plan.w_self[i];
+        const float4 self = stepped(i);
+        float4 acc = make_float4(ws * self.x, ws * self.y, ws * self.z, ws * self.w);
+        const int cnt = plan.cnt[i];
+        for (int k = 0; k < cnt; ++k)
+            acc = fma4(plan.w[(size_t)i * plan.stride + k], stepped(plan.idx[(size_t)i * plan.stride + k]), acc);
+        if (mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
+        *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
+    }
+}
+
+int auto_group_size(const dbw_handle* h) {
+    if (h->mix_panel_cols < 0) return 0;  // direct kernel forced
+    if (h->mix_panel_cols) return ((size_t)h->N * h->mix_panel_cols * 4 <= (size_t)h->smem_optin) ? h->mix_panel_cols / 4 : 0;
+    // widest panel whose staging buffer still lets two CTAs share an SM
+    const size_t budget = (size_t)(h->smem_optin) / 2 - 1024;
+    for (int gs = 32; gs >= 4; gs >>= 1)
+        if ((size_t)h->N * gs * 16 <= budget) return gs;
+    return ((size_t)h->N * 4 * 16 <= (size_t)h->smem_optin) ? 4 : 0;
+}
+
+template <int GS>
+int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+                 cudaStream_t s) {
+    const size_t smem = (size_t)h->N * GS * 16;
+    static bool configured[64] = {};
+    if (!configured[h->device & 63]) {
+        DBW_CUDA(cudaFuncSetAttribute(mix_panel_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      h->smem_optin));
+        configured[h->device & 63] = true;
+    }
+    int per_sm = 0;
+    DBW_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mix_panel_kernel<GS>, kMixThreads, smem));
+    if (per_sm < 1) return DBW_ERR_BAD_SHAPE;
+    const int n_panels = (int)((h->ld + 4 * GS - 1) / (4 * GS));
+    const int grid = n_panels < per_sm * h->sm_count ? n_panels : per_sm * h->sm_count;
+    mix_panel_kernel<GS><<<grid, kMixThreads, smem, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, h->plan,
+                                                        (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0,
+                                                        n_panels);
+    DBW_LAUNCHED();
+    return DBW_OK;
+}
+
+}  // namespace
+
+bool mix_panel_fits(const dbw_handle* h) { return auto_group_size(h) != 0; }
+
+int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+               cudaStream_t s) {
+    switch (auto_group_size(h)) {
+        case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, s);
+        case 16: return launch_panel<16>(h, X, G, lr, lr_pw, X_out, s);
+        case 8: return launch_panel<8>(h, X, G, lr, lr_pw, X_out, s);
+        case 4: return launch_panel<4>(h, X, G, lr, lr_pw, X_out, s);
+        default: break;
+    }
+    if (X_out == X) return DBW_ERR_BAD_SHAPE;
+    const long long total = (long long)h->N * (h->ld / 4);
+    long long blocks = (total + 255) / 256;
+    const long long cap = (long long)h->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    mix_direct_kernel<<<(int)blocks, 256, 0, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, h->plan,
+                                                 (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0);
+    DBW_LAUNCHED();
+    return DBW_OK;
+}
+
+}  // namespace dbw

@@ -1,0 +1,200 @@
+"""GPU parity on the five workloads (whole rounds through dbw_round / dbw_update_backups).
+
+Every round is checked teacher-forced: the GPU round starts from the oracle's current fp32
+parameters, so the 1e-5 per-round bar of the fp32 path is not blurred by drift.  A free-running
+GPU trajectory is carried alongside and compared at the end with the looser bar stated per test.
+Masks, times, b and theta never depend on the parameters and are bit-exact on every round.
+"""
+import numpy as np
+import pytest
+
+from oracle import dbw_oracle as orc
+from workloads import configs as wl
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def row_rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    num = np.abs(got - ref).max(axis=1)
+    den = np.maximum(np.abs(ref).max(axis=1), 1e-30)
+    return float((num / den).max())
+
+
+class Sim:
+    """One workload on both sides: the oracle in float64 and the GPU library."""
+
+    def __init__(self, w, gemm_flag=0):
+        import paper_2102_06280_b200 as p
+        self.p, self.w = p, w
+        self.m = p.model_layout(w.layers, w.batch)
+        flags = gemm_flag | (p.WEIGHT_UNIFORM if w.weight_rule == "uniform" else 0)
+        self.h = p.Dbw(w.rowptr, w.col, d=self.m.d, model=self.m, flags=flags)
+        means = wl.class_means(w)
+        data = [wl.worker_dataset(w, i, means) for i in range(w.N)]
+        self.feat = np.stack([f for f, _ in data])
+        self.labels = np.stack([l for _, l in data])
+        self.h.set_dataset(dev(self.feat), dev(self.labels), w.samples)
+        self.X0 = np.stack([wl.init_params(w, i) for i in range(w.N)])
+        self.dtur_ref = orc.Dtur(w.rowptr, w.col)
+        n, nnz = w.N, len(w.col)
+        self.kept = torch.zeros(nnz, dtype=torch.uint8, device="cuda")
+        self.Tw = torch.zeros(n, dtype=torch.float64, device="cuda")
+        self.Tn = torch.zeros(n, dtype=torch.float64, device="cuda")
+        self.Tr = torch.zeros(1, dtype=torch.float64, device="cuda")
+        self.loss = torch.zeros(n, device="cuda")
+        self.b_d = torch.zeros(n, dtype=torch.int32, device="cuda")
+        self.th = torch.zeros(1, dtype=torch.float64, device="cuda")
+
+    def backups(self, k, t):
+        """b for round k on both sides (bit-exact check included)."""
+        w = self.w
+        if w.backups == "fixed":
+            b = wl.fixed_backups(w)
+            self.b_d.copy_(dev(b))
+            return b
+        if k == 0:                      # Algorithm 1: the first iteration waits for every neighbour
+            b = np.zeros(w.N, dtype=np.int32)
+            self.b_d.zero_()
+            return b
+        b, theta = self.dtur_ref.update_backups(t)
+        self.h.update_backups(dev(t), self.b_d, self.th)
+        assert np.array_equal(self.b_d.cpu().numpy(), b) and float(self.th.cpu()[0]) == theta
+        self.theta = theta
+        return b
+
+    def gpu_round(self, X_d, t, idx, out_d):
+        self.h.round(X_d, dev(t), self.b_d, self.w.lr, out_d, self.kept, batch_idx=dev(idx),
+                     T_worker=self.Tw, T_nbr=self.Tn, T_round=self.Tr, loss=self.loss)
+        torch.cuda.synchronize()
+
+    def oracle_round(self, X, t, b, idx):
+        w = self.w
+        feats = [self.feat[i][idx[i]] for i in range(w.N)]
+        labels = [self.labels[i][idx[i]] for i in range(w.N)]
+        return orc.dbw_round(w.rowptr, w.col, X, t, b, w.lr, layers=w.layers, feats=feats, labels=labels,
+                             rule=w.weight_rule)
+
+    def check_discrete(self, r):
+        assert np.array_equal(self.kept.cpu().numpy(), r["kept"])
+        assert np.array_equal(self.Tn.cpu().numpy(), r["T_nbr"])
+        assert np.array_equal(self.Tw.cpu().numpy(), r["T_worker"])
+        assert float(self.Tr.cpu()[0]) == r["T_round"]
+
+
+def _run(w, rounds, param_rounds, gemm_flag=0, tol_round=1e-5, tol_free=None):
+    sim = Sim(w, gemm_flag)
+    m = sim.m
+    times = wl.arrival_times(w, rounds)
+    X_ref = sim.X0.astype(np.float64)           # oracle trajectory, rounded to fp32 each round (teacher)
+    X_free = dev(m.pack(sim.X0))                # GPU free-running trajectory
+    X_orc_free = sim.X0.astype(np.float64)      # oracle free-running trajectory in float64
+    out = torch.empty_like(X_free)
+    worst = 0.0
+    for k in range(rounds):
+        t = times[k]
+        b = sim.backups(k, t)
+        idx = wl.batch_indices(w, k)
+        if k < param_rounds:
+            # teacher-forced: both sides start from the same fp32 parameters
+            X32 = X_ref.astype(np.float32)
+            r = sim.oracle_round(X32, t, b, idx)
+            sim.gpu_round(dev(m.pack(X32)), t, idx, out)
+            sim.check_discrete(r)
+            got = m.unpack(out.cpu().numpy())
+            err = row_rel_err(got, r["X"])
+            worst = max(worst, err)
+            assert err <= tol_round, (k, err)
+            assert np.abs(sim.loss.cpu().numpy() - r["loss"]).max() <= 1e-3 * max(1.0, np.abs(r["loss"]).max())
+            assert not np.any(m.pack(got) != out.cpu().numpy())      # padding stays zero
+            X_ref = r["X"]
+            # free-running on both sides
+            if tol_free is not None:
+                X_orc_free = sim.oracle_round(X_orc_free, t, b, idx)["X"]
+                sim.gpu_round(X_free, t, idx, X_free)                 # in place
+        else:
+            # discrete outputs only: selection / times never read the parameters
+            kept = orc.select_fastest(w.rowptr, w.col, t, b)
+            Tn, Tw, Tr = orc.round_times(w.rowptr, w.col, t, b, kept)
+            sim.h.select(dev(t), sim.b_d, sim.kept, sim.Tw, sim.Tn, sim.Tr)
+            torch.cuda.synchronize()
+            sim.check_discrete(dict(kept=kept, T_nbr=Tn, T_worker=Tw, T_round=Tr))
+        if w.backups == "dtur" and k > 0:
+            assert float(sim.Tr.cpu()[0]) == sim.theta                # the round lasts exactly theta
+    if tol_free is not None:
+        err = row_rel_err(m.unpack(X_free.cpu().numpy()), X_orc_free)
+        assert err <= tol_free, err
+    assert sim.h.status() == 0
+    sim.h.close()
+    return worst
+
+
+def test_config0_all_rounds():
+    w = wl.make_workload(0)
+    _run(w, w.rounds, w.rounds, tol_round=1e-5, tol_free=1e-4)
+
+
+def test_config1_dynamic_backups():
+    w = wl.make_workload(1)
+    _run(w, w.rounds, 12, tol_round=1e-5, tol_free=1e-4)
+
+
+def test_config4_reduced_width():
+    """Config 4's graph, backups, weights and value distributions at d = 8192 (+ ragged tail)."""
+    import paper_2102_06280_b200 as p
+    w = wl.make_workload(4, d=8192 + 36)
+    n, d = w.N, w.d
+    h = p.Dbw(w.rowptr, w.col, d=d, flags=p.WEIGHT_UNIFORM)
+    X = wl.gaussian_rows(w.init_seed, range(n), d)
+    G = wl.gaussian_rows(wl.external_gradient_seed(w), range(n), d, scale=0.01)
+    times = wl.arrival_times(w)
+    bs = wl.uniform_backups(w)
+    Xd, Gd = dev(X), dev(G)
+    kept = torch.zeros(len(w.col), dtype=torch.uint8, device="cuda")
+    Tw = torch.zeros(n, dtype=torch.float64, device="cuda")
+    Tr = torch.zeros(1, dtype=torch.float64, device="cuda")
+    Xref = X.astype(np.float64)
+    for k in range(w.rounds):
+        r = orc.dbw_round(w.rowptr, w.col, Xref.astype(np.float32), times[k], bs[k], w.lr, G=G, rule=orc.UNIFORM)
+        Xin = dev(Xref.astype(np.float32))
+        h.round(Xin, dev(times[k]), dev(bs[k]), w.lr, Xin, kept, G_ext=Gd, T_worker=Tw, T_round=Tr)
+        torch.cuda.synchronize()
+        assert np.array_equal(kept.cpu().numpy(), r["kept"])
+        assert np.array_equal(Tw.cpu().numpy(), r["T_worker"]) and float(Tr.cpu()[0]) == r["T_round"]
+        assert row_rel_err(Xin.cpu().numpy(), r["X"]) <= 1e-5
+        Xref = r["X"]
+    assert h.status() == 0
+    h.close()
+
+
+def test_round_host_matches_device_round():
+    """dbw_round_host (per-round inputs in pinned host memory) == dbw_round."""
+    w = wl.make_workload(0)
+    sim = Sim(w)
+    m = sim.m
+    t = wl.arrival_times(w, 1)[0]
+    b = wl.fixed_backups(w)
+    idx = wl.batch_indices(w, 0)
+    Xd = dev(m.pack(sim.X0))
+    out1, out2 = torch.empty_like(Xd), torch.empty_like(Xd)
+    sim.b_d.copy_(dev(b))
+    sim.gpu_round(Xd, t, idx, out1)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_t, h_b, h_idx = pin(t), pin(b), pin(idx)
+    h_kept = torch.zeros(len(w.col), dtype=torch.uint8).pin_memory()
+    h_Tw = torch.zeros(w.N, dtype=torch.float64).pin_memory()
+    h_Tr = torch.zeros(1, dtype=torch.float64).pin_memory()
+    h_loss = torch.zeros(w.N).pin_memory()
+    sim.h.round_host(Xd, h_t, h_b, w.lr, out2, h_batch_idx=h_idx, h_kept=h_kept, h_T_worker=h_Tw, h_T_round=h_Tr,
+                     h_loss=h_loss)
+    torch.cuda.synchronize()
+    assert torch.equal(out1, out2)
+    assert torch.equal(h_kept, sim.kept.cpu()) and torch.equal(h_Tw, sim.Tw.cpu()) and torch.equal(h_Tr, sim.Tr.cpu())
+    assert torch.equal(h_loss, sim.loss.cpu())
+    sim.h.close()

@@ -1,0 +1,235 @@
+"""GPU parity, kernel by kernel, through the C ABI against the CPU oracle on the same seeded inputs.
+
+Bars: kept masks, T_nbr / T_worker / T_round, b and theta are bit-exact (only comparisons touch
+the times); parameters after the fp32 mix agree to 1e-5 per row (max-norm relative), which
+leaves two orders of magnitude over the fp32 rounding of a <= 40-term weighted sum.
+"""
+import numpy as np
+import pytest
+
+from oracle import dbw_oracle as orc
+from workloads import configs as wl
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _dbw():
+    import paper_2102_06280_b200 as p
+    return p
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def row_rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    num = np.abs(got - ref).max(axis=1)
+    den = np.maximum(np.abs(ref).max(axis=1), 1e-30)
+    return float((num / den).max())
+
+
+GRAPHS = {
+    "ring8": lambda: wl.ring(8),
+    "path2": lambda: wl.path(2),
+    "complete40": lambda: wl.complete(40),          # degree 39 > one warp
+    "complete70": lambda: wl.complete(70),          # degree 69: three 32-neighbour chunks
+    "reg4_32": lambda: wl.random_regular(32, 4, 2),
+    "er64": lambda: wl.erdos_renyi_connected(64, 0.2, 3),
+    "reg32_256": lambda: wl.random_regular(256, 32, 11),
+    "star_like": lambda: wl._csr_from_edges(6, [(0, 1), (0, 2), (0, 3), (0, 4), (0, 5)]),  # degree-1 leaves
+}
+
+
+def _select_gpu(h, n, nnz, t, b):
+    kept = torch.zeros(nnz, dtype=torch.uint8, device="cuda")
+    Tw = torch.zeros(n, dtype=torch.float64, device="cuda")
+    Tn = torch.zeros(n, dtype=torch.float64, device="cuda")
+    Tr = torch.zeros(1, dtype=torch.float64, device="cuda")
+    h.select(dev(t), dev(b.astype(np.int32)), kept, Tw, Tn, Tr)
+    torch.cuda.synchronize()
+    return kept.cpu().numpy(), Tw.cpu().numpy(), Tn.cpu().numpy(), float(Tr.cpu()[0])
+
+
+@pytest.mark.parametrize("name", list(GRAPHS))
+def test_selection_bit_exact(name):
+    p = _dbw()
+    rowptr, col = GRAPHS[name]()
+    n = len(rowptr) - 1
+    deg = np.diff(rowptr)
+    h = p.Dbw(rowptr, col, d=4)
+    rng = np.random.default_rng(5)
+    cases = []
+    for trial in range(6):
+        t = 1.0 + rng.exponential(1.0, size=n)
+        if trial % 2:                                  # engineered ties
+            t = np.round(t * 2) / 2
+        cases.append((t, rng.integers(0, deg + 1)))
+    cases.append((1.0 + rng.exponential(1.0, size=n), np.zeros(n, dtype=np.int64)))   # b = 0
+    cases.append((1.0 + rng.exponential(1.0, size=n), deg.copy()))                     # b = deg
+    cases.append((np.ones(n), rng.integers(0, deg + 1)))                               # all times equal
+    for t, b in cases:
+        kept, Tw, Tn, Tr = _select_gpu(h, n, len(col), t, b)
+        ref = orc.select_fastest(rowptr, col, t, b)
+        assert np.array_equal(kept, ref)
+        rTn, rTw, rTr = orc.round_times(rowptr, col, t, b, ref)
+        assert np.array_equal(Tn, rTn) and np.array_equal(Tw, rTw) and Tr == rTr
+    assert h.status() == 0
+    h.close()
+
+
+def test_selection_flags_bad_inputs():
+    p = _dbw()
+    rowptr, col = wl.ring(8)
+    h = p.Dbw(rowptr, col, d=4)
+    t = np.arange(8, dtype=np.float64)
+    b = np.array([0, 5, 0, -2, 0, 0, 0, 0])
+    kept, *_ = _select_gpu(h, 8, len(col), t, b)
+    assert h.status() & p.STATUS_BAD_B
+    ref = orc.select_fastest(rowptr, col, t, np.clip(b, 0, 2))      # clamped, not trapped
+    assert np.array_equal(kept, ref)
+    t[3] = np.nan
+    kept, *_ = _select_gpu(h, 8, len(col), t, np.ones(8, dtype=np.int64))
+    assert h.status() & p.STATUS_NAN_TIME
+    t[3] = np.inf                                                    # NaN is ordered last
+    assert np.array_equal(kept, orc.select_fastest(rowptr, col, t, np.ones(8, dtype=np.int64)))
+    assert h.status() == 0
+    h.close()
+
+
+@pytest.mark.parametrize("name,d", [("ring8", 7850), ("reg4_32", 1000), ("er64", 4100), ("complete40", 260),
+                                     ("reg32_256", 3000)])
+@pytest.mark.parametrize("rule", ["metropolis", "uniform"])
+@pytest.mark.parametrize("order", ["local_then_mix", "mix_then_correct"])
+def test_mix_matches_oracle(name, d, rule, order):
+    p = _dbw()
+    rowptr, col = GRAPHS[name]()
+    n = len(rowptr) - 1
+    deg = np.diff(rowptr)
+    ld = (d + 3) // 4 * 4
+    flags = (p.WEIGHT_UNIFORM if rule == "uniform" else 0) | (p.ORDER_MIX_THEN_CORRECT if order == "mix_then_correct" else 0)
+    h = p.Dbw(rowptr, col, d=d, ld=ld, flags=flags)
+    rng = np.random.default_rng(8)
+    X = np.zeros((n, ld), dtype=np.float32)
+    G = np.zeros((n, ld), dtype=np.float32)
+    X[:, :d] = rng.standard_normal((n, d), dtype=np.float32)
+    G[:, :d] = rng.standard_normal((n, d), dtype=np.float32)
+    t = 1.0 + rng.exponential(1.0, size=n)
+    b = rng.integers(0, deg + 1)
+    b[0] = deg[0]                                         # one worker waits for nobody
+    kept = orc.select_fastest(rowptr, col, t, b)
+    ws, we = orc.mixing_weights(rowptr, col, b, kept, rule)
+    ref = orc.mix_update(rowptr, col, X, G, ws, we, 0.05, order)
+    Xd, Gd, kd, bd = dev(X), dev(G), dev(kept), dev(b.astype(np.int32))
+    for panel in (0, 16, 32, 64, 128, -1):
+        h.set_mix_panel(panel)
+        out = torch.full_like(Xd, float("nan"))
+        h.mix(Xd, Gd, kd, bd, 0.05, out)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        assert row_rel_err(got, ref) <= 1e-5, panel
+        assert not np.any(got[:, d:])                      # padding stays zero
+        if panel != -1 and h.mix_in_place_ok():
+            inpl = Xd.clone()
+            h.mix(inpl, Gd, kd, bd, 0.05, inpl)
+            torch.cuda.synchronize()
+            assert np.array_equal(inpl.cpu().numpy(), got)  # in place == out of place, bit for bit
+    # per-worker learning rates (eta_j of Eq. 4)
+    lrw = (0.01 + 0.1 * rng.random(n)).astype(np.float32)
+    h.set_mix_panel(0)
+    out = torch.empty_like(Xd)
+    h.mix(Xd, Gd, kd, bd, 0.0, out, lr_per_worker=dev(lrw))
+    torch.cuda.synchronize()
+    ref = orc.mix_update(rowptr, col, X, G, ws, we, lrw.astype(np.float64), order)
+    assert row_rel_err(out.cpu().numpy(), ref) <= 1e-5
+    assert h.status() == 0
+    h.close()
+
+
+def test_mix_rejects_bad_aliasing():
+    p = _dbw()
+    rowptr, col = wl.ring(8)
+    h = p.Dbw(rowptr, col, d=64)
+    X = torch.zeros(8 * 64 + 64, device="cuda")
+    G = torch.zeros(8 * 64, device="cuda")
+    kept = torch.ones(16, dtype=torch.uint8, device="cuda")
+    b = torch.zeros(8, dtype=torch.int32, device="cuda")
+    with pytest.raises(p.DbwError):
+        h.mix(X[:512], G, kept, b, 0.1, X[32:544])          # partial overlap
+    with pytest.raises(p.DbwError):
+        h.mix(X[:512], G, kept, b, 0.1, G)                  # output over the gradients
+    h.set_mix_panel(-1)
+    with pytest.raises(p.DbwError):
+        h.mix(X[:512], G, kept, b, 0.1, X[:512])            # direct kernel cannot run in place
+    h.close()
+
+
+@pytest.mark.parametrize("name", ["ring8", "reg4_32", "er64", "complete40"])
+def test_update_backups_bit_exact_and_resume(name):
+    p = _dbw()
+    rowptr, col = GRAPHS[name]()
+    n = len(rowptr) - 1
+    h = p.Dbw(rowptr, col, d=4)
+    assert np.array_equal(h.links(), np.array(orc.spanning_links(rowptr, col)))
+    ref = orc.Dtur(rowptr, col)
+    rng = np.random.default_rng(3)
+    b_d = torch.zeros(n, dtype=torch.int32, device="cuda")
+    th_d = torch.zeros(1, dtype=torch.float64, device="cuda")
+    rounds = 2 * (n - 1) + 3
+    times = 1.0 + rng.exponential(1.0, size=(rounds, n))
+    times[1] = np.round(times[1])                            # ties between links
+    blob = None
+    for k in range(rounds):
+        if k == n // 2:
+            blob = h.state_export()
+            saved = (list(ref.covered), ref.step)
+        h.update_backups(dev(times[k]), b_d, th_d)
+        torch.cuda.synchronize()
+        rb, rtheta = ref.update_backups(times[k])
+        assert np.array_equal(b_d.cpu().numpy(), rb) and float(th_d.cpu()[0]) == rtheta
+    # resume from the saved state reproduces the same sequence
+    h.state_import(blob)
+    ref.covered, ref.step = saved
+    for k in range(n // 2, n // 2 + 5):
+        h.update_backups(dev(times[k]), b_d, th_d)
+        rb, rtheta = ref.update_backups(times[k])
+        assert np.array_equal(b_d.cpu().numpy(), rb) and float(th_d.cpu()[0]) == rtheta
+    h.reset_backups()
+    fresh = orc.Dtur(rowptr, col)
+    h.update_backups(dev(times[0]), b_d, th_d)
+    assert np.array_equal(b_d.cpu().numpy(), fresh.update_backups(times[0])[0])
+    with pytest.raises(p.DbwError):
+        h.state_import(blob[:-4])
+    h.close()
+
+
+@pytest.mark.parametrize("dims,batch,n", [([784, 10], 32, 8), ([20, 13, 7], 5, 3), ([100, 70, 33, 10], 19, 4),
+                                           ([784, 200, 10], 64, 6)])
+def test_grad_fp32_matches_oracle(dims, batch, n):
+    p = _dbw()
+    rowptr, col = wl.ring(max(n, 3)) if n >= 3 else wl.path(n)
+    n = len(rowptr) - 1
+    m = p.model_layout(dims, batch)
+    h = p.Dbw(rowptr, col, d=m.d, model=m)
+    rng = np.random.default_rng(0)
+    S = 3 * batch
+    feat = rng.random((n, S, dims[0]), dtype=np.float32)
+    labels = rng.integers(0, dims[-1], size=(n, S)).astype(np.int32)
+    Xl = (rng.standard_normal((n, m.d)) * 0.2).astype(np.float32)
+    idx = np.stack([rng.permutation(S)[:batch] for _ in range(n)]).astype(np.int32)
+    h.set_dataset(dev(feat), dev(labels), S)
+    G = torch.zeros(n, m.ld, device="cuda")
+    loss = torch.zeros(n, device="cuda")
+    h.grad(dev(m.pack(Xl)), dev(idx), G, loss)
+    torch.cuda.synchronize()
+    got = m.unpack(G.cpu().numpy())
+    for i in range(n):
+        g, l = orc.mlp_grad(Xl[i], dims, feat[i][idx[i]], labels[i][idx[i]])
+        assert np.abs(got[i] - g).max() <= 1e-5 * max(np.abs(g).max(), 1e-30)
+        assert abs(float(loss[i]) - l) <= 1e-5 * max(abs(l), 1.0)
+    Gp = G.cpu().numpy()
+    assert np.count_nonzero(Gp) == np.count_nonzero(got)      # padding untouched
+    assert h.status() == 0
+    h.close()
