@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the cb-DyBW round: simulated worker-rounds/s on one B200 (replicas on N GPUs).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+A step is one round of the whole hot path over one batch of synthetic input: backup counts
+(threshold rule, where the workload is dynamic), mini-batch gradients (where the workload has a
+model), fastest-neighbour selection, weights, fused mix + SGD.  One JSON line is printed by
+rank 0.  `value` is timed with everything resident in HBM; `e2e` is the same loop through
+dbw_round_host with the per-round inputs in pinned host memory and the per-round results read
+back.  `roofline` is the mix kernel: 12 bytes per parameter element (read x, read g, write x')
+over its own CUDA-event time inside the timed loop, against the measured copy bandwidth.
+`cpu_baseline` times the double-precision CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import configs as wl  # noqa: E402
+
+METRIC = "simulated worker-rounds/sec"
+UNIT = "worker-rounds/s"
+DEFAULT_CONFIG = 4
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# workload set-up shared by the bench and the full-size parity tests
+# ------------------------------------------------------------------------------------------
+
+class Job:
+    """One workload resident on one GPU, stepped through the C ABI."""
+
+    def __init__(self, config: int, device: int = 0, rounds: int | None = None, **overrides):
+        import torch
+        import paper_2102_06280_b200 as p
+        self.torch, self.p = torch, p
+        torch.cuda.set_device(device)
+        self.dev = torch.device("cuda", device)
+        w = self.w = wl.make_workload(config, **overrides)
+        self.n_rounds = rounds or w.rounds
+        flags = (p.WEIGHT_UNIFORM if w.weight_rule == "uniform" else 0) | (p.GEMM_BF16 if w.precision == "bf16" else 0)
+        if w.layers is not None:
+            self.m = p.model_layout(w.layers, w.batch)
+            self.h = p.Dbw(w.rowptr, w.col, d=self.m.d, model=self.m, flags=flags, device=device)
+            means = wl.class_means(w)
+            feat = torch.empty((w.N, w.samples, w.layers[0]), dtype=torch.float32, device=self.dev)
+            labels = torch.empty((w.N, w.samples), dtype=torch.int32, device=self.dev)
+            for i in range(w.N):
+                f, l = wl.worker_dataset(w, i, means)
+                feat[i].copy_(torch.from_numpy(f))
+                labels[i].copy_(torch.from_numpy(l))
+            self.feat, self.labels = feat, labels
+            self.h.set_dataset(feat, labels, w.samples)
+            X0 = np.stack([wl.init_params(w, i) for i in range(w.N)])
+            self.X = torch.from_numpy(self.m.pack(X0)).to(self.dev)
+            self.G = None
+            self.h_idx = torch.from_numpy(np.stack([wl.batch_indices(w, k) for k in range(self.n_rounds)])).pin_memory()
+            self.d_idx = self.h_idx.to(self.dev)
+            self.ld = self.m.ld
+        else:
+            self.m = None
+            self.ld = w.d
+            self.h = p.Dbw(w.rowptr, w.col, d=w.d, ld=w.d, flags=flags, device=device)
+            self.X = torch.empty((w.N, w.d), dtype=torch.float32, device=self.dev)
+            self.G = torch.empty((w.N, w.d), dtype=torch.float32, device=self.dev)
+            step = 64
+            for r0 in range(0, w.N, step):
+                rows = range(r0, min(w.N, r0 + step))
+                self.X[r0:r0 + step].copy_(torch.from_numpy(wl.gaussian_rows(w.init_seed, rows, w.d)))
+                self.G[r0:r0 + step].copy_(torch.from_numpy(
+                    wl.gaussian_rows(wl.external_gradient_seed(w), rows, w.d, scale=0.01)))
+            self.h_idx = self.d_idx = None
+        self.h_t = torch.from_numpy(wl.arrival_times(w, self.n_rounds)).pin_memory()
+        self.d_t = self.h_t.to(self.dev)
+        if w.backups == "fixed":
+            hb = np.tile(wl.fixed_backups(w), (self.n_rounds, 1))
+        elif w.backups == "uniform":
+            hb = wl.uniform_backups(w, self.n_rounds)
+        else:
+            hb = np.zeros((self.n_rounds, w.N), dtype=np.int32)     # round 1: everyone waits for everyone
+        self.h_b = torch.from_numpy(np.ascontiguousarray(hb)).pin_memory()
+        self.d_b = self.h_b.to(self.dev)
+        n, nnz = w.N, len(w.col)
+        self.kept = torch.zeros(nnz, dtype=torch.uint8, device=self.dev)
+        self.Tw = torch.zeros(n, dtype=torch.float64, device=self.dev)
+        self.Tr = torch.zeros(1, dtype=torch.float64, device=self.dev)
+        self.loss = torch.zeros(n, dtype=torch.float32, device=self.dev)
+        self.b_dyn = torch.zeros(n, dtype=torch.int32, device=self.dev)
+        self.hk = torch.zeros(nnz, dtype=torch.uint8).pin_memory()
+        self.hTw = torch.zeros(n, dtype=torch.float64).pin_memory()
+        self.hTr = torch.zeros(1, dtype=torch.float64).pin_memory()
+        self.hloss = torch.zeros(n, dtype=torch.float32).pin_memory()
+        self.hb_out = torch.zeros(n, dtype=torch.int32).pin_memory()
+        self.k = 0
+        torch.cuda.synchronize()
+
+    def step(self):
+        """One round, every input already on the device (in place on X)."""
+        w, r = self.w, self.k % self.n_rounds
+        b = self.d_b[r]
+        if w.backups == "dtur" and self.k > 0:
+            self.h.update_backups(self.d_t[r], self.b_dyn)
+            b = self.b_dyn
+        self.h.round(self.X, self.d_t[r], b, w.lr, self.X, self.kept,
+                     batch_idx=None if self.d_idx is None else self.d_idx[r], G_ext=self.G,
+                     T_worker=self.Tw, T_round=self.Tr, loss=self.loss)
+        self.k += 1
+
+    def step_host(self):
+        """One round with the per-round inputs in pinned host memory and the results read back."""
+        w, r = self.w, self.k % self.n_rounds
+        dyn = w.backups == "dtur" and self.k > 0
+        self.h.round_host(self.X, self.h_t[r], None if dyn else self.h_b[r], w.lr, self.X,
+                          h_batch_idx=None if self.h_idx is None else self.h_idx[r], G_ext=self.G,
+                          h_kept=self.hk, h_T_worker=self.hTw, h_T_round=self.hTr,
+                          h_loss=None if self.h_idx is None else self.hloss, h_b_out=self.hb_out if dyn else None)
+        self.torch.cuda.current_stream().synchronize()      # the caller reads the round's results
+        self.k += 1
+
+    def host_bytes_per_step(self):
+        w = self.w
+        h2d = w.N * 8 + (0 if w.backups == "dtur" else w.N * 4) + (0 if self.h_idx is None else w.N * w.batch * 4)
+        d2h = len(w.col) + w.N * 8 + 8 + (0 if self.h_idx is None else w.N * 4) + (w.N * 4 if w.backups == "dtur" else 0)
+        return h2d, d2h
+
+    def mix_bytes_per_launch(self):
+        return 12 * self.w.N * self.ld
+
+    def close(self):
+        self.h.close()
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.device, self.proc, self.path = device, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.device), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle timing (baseline leg and the reference arm)
+# ------------------------------------------------------------------------------------------
+
+def oracle_sample_seconds(w, k: int = 0, budget_s: float = 12.0):
+    """Times the oracle on a bounded sample of round k; returns (estimated s per full round, description).
+
+    Selection, times, weights (and the threshold rule) run whole.  Gradients run for a few
+    workers and scale by N / sampled.  The mix runs on all rows x a block of columns and scales
+    by d / sampled columns (the update is independent per column).
+    """
+    from oracle import dbw_oracle as orc
+    rng = np.random.default_rng(123)
+    t = wl.arrival_times(w, max(k + 1, 2))[k]
+    t0 = time.perf_counter()
+    if w.backups == "dtur":
+        b, _ = orc.Dtur(w.rowptr, w.col).update_backups(t)
+    elif w.backups == "uniform":
+        b = wl.uniform_backups(w, k + 1)[k]
+    else:
+        b = wl.fixed_backups(w)
+    kept = orc.select_fastest(w.rowptr, w.col, t, b)
+    orc.round_times(w.rowptr, w.col, t, b, kept)
+    ws, we = orc.mixing_weights(w.rowptr, w.col, b, kept, w.weight_rule)
+    t_discrete = time.perf_counter() - t0
+    t_grad, n_grad = 0.0, 0
+    if w.layers is not None:
+        means = wl.class_means(w)
+        idx = wl.batch_indices(w, k)
+        while n_grad < w.N and t_grad < budget_s / 2:
+            i = n_grad
+            f, l = wl.worker_dataset(w, i, means)
+            x = wl.init_params(w, i)
+            t0 = time.perf_counter()
+            orc.mlp_grad(x, w.layers, f[idx[i]], l[idx[i]])
+            t_grad += time.perf_counter() - t0
+            n_grad += 1
+        t_grad_full = t_grad * w.N / n_grad
+    else:
+        t_grad_full = 0.0
+    cols = 1024
+    t_mix, t_mix_full = 0.0, 0.0
+    while True:
+        cols = min(cols, w.d)
+        X = rng.standard_normal((w.N, cols)).astype(np.float32)
+        G = (0.01 * rng.standard_normal((w.N, cols))).astype(np.float32)
+        t0 = time.perf_counter()
+        orc.mix_update(w.rowptr, w.col, X, G, ws, we, w.lr)
+        t_mix = time.perf_counter() - t0
+        t_mix_full = t_mix * w.d / cols
+        if cols == w.d or t_mix > budget_s / 4:
+            break
+        cols *= 4
+    desc = ("round %d: selection/times/weights%s whole (%.3fs); gradients of %d of %d workers (%.2fs, scaled); "
+            "mix on all %d rows x %d of %d columns (%.2fs, scaled)" %
+            (k, "/threshold rule" if w.backups == "dtur" else "", t_discrete, n_grad, w.N, t_grad, w.N, cols, w.d, t_mix))
+    return t_discrete + t_grad_full + t_mix_full, desc
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.make_workload(args.config)
+    # the whole run (warm-up included) is bounded to about two minutes of CPU work
+    budget = min(args.ref_budget, 120.0 / (args.steps + args.warmup))
+    for _ in range(args.warmup):
+        oracle_sample_seconds(w, 0, budget_s=budget)
+    est = []
+    desc = ""
+    for k in range(args.steps):
+        s, desc = oracle_sample_seconds(w, k % w.rounds, budget_s=budget)
+        est.append(s)
+    sec = float(np.mean(est))
+    value = w.N / sec
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "N": w.N, "d": w.d, "note": "CPU oracle, each step a bounded sample scaled to a full round"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# the GPU arm
+# ------------------------------------------------------------------------------------------
+
+def timed_loop(job, steps, fn, dist):
+    import torch
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tt = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    return ms
+
+
+def run_ours(args):
+    import torch
+    from paper_2102_06280_b200 import build, binding
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        torch.cuda.set_device(local)
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    if rank == 0:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+    job = Job(args.config, device=local)
+    w = job.w
+    for _ in range(args.warmup):
+        job.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    job.h.profile(True)
+    job.h.profile_read()
+    launches0 = binding.launch_count()
+    ms = timed_loop(job, args.steps, job.step, dist)
+    launches = binding.launch_count() - launches0
+    stage_ms, stage_rounds = job.h.profile_read()
+    job.h.profile(False)
+    # end to end: per-round inputs from pinned host memory, results read back every round
+    for _ in range(min(args.warmup, 3)):
+        job.step_host()
+    ms_e2e = timed_loop(job, args.steps, job.step_host, dist)
+    clocks = sampler.stop() if rank == 0 else None
+    status = job.h.status()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks, peak_kind = measured_peaks()
+    value = world * w.N * args.steps / (ms * 1e-3)
+    e2e = world * w.N * args.steps / (ms_e2e * 1e-3)
+    h2d, d2h = job.host_bytes_per_step()
+    mix_ms = stage_ms["mix"] / max(stage_rounds, 1)
+    achieved = job.mix_bytes_per_launch() / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
+    roofline = {"kernel": "mix_panel_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind,
+                "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
+                "bytes_per_launch": job.mix_bytes_per_launch(), "ms_per_launch": mix_ms}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32" if w.precision == "fp32" else "bf16xbf16->f32 GEMM, f32 mix",
+            "data": "synthetic",
+            "config": {"workload": w.name, "N": w.N, "d": w.d, "ld": job.ld, "nnz": int(len(w.col)),
+                       "batch": w.batch, "layers": w.layers, "backups": w.backups, "weights": w.weight_rule,
+                       "l2": "inputs larger than L2 (X and G each %.2f GB)" % (w.N * job.ld * 4 / 1e9)
+                             if w.N * job.ld * 4 > 126e6 else "working set smaller than L2: cache-resident by design",
+                       "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+            "stage_ms": {k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks, "device_status": status}
+    if not args.no_cpu_baseline and world == 1:
+        sec, desc = oracle_sample_seconds(w, 0, budget_s=args.ref_budget)
+        line["cpu_baseline"] = {"value": w.N / sec, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc}
+    print(json.dumps(line))
+    job.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU oracle work per sampled step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -147,13 +147,15 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
  * The same round for callers whose per-round inputs live in HOST memory (pinned memory makes
  * the copies asynchronous).  X / X_out / G_ext stay DEVICE (the parameters are the state of the
  * simulation); h_t[N], h_b[N], h_batch_idx[N][batch] are copied to the device on `stream`, the
- * round runs, and h_kept[nnz], h_T_worker[N], h_T_round[1], h_loss[N] (each nullable) are copied
- * back on `stream`.  The call does not synchronise.
+ * round runs, and h_kept[nnz], h_T_worker[N], h_T_round[1], h_loss[N], h_b_out[N] (each
+ * nullable) are copied back on `stream`.  When h_b is NULL the backup counts come from the
+ * threshold rule: dbw_update_backups runs on the copied times first (Algorithm 2 feeding
+ * Algorithm 1) and h_b_out receives them.  The call does not synchronise.
  */
 int dbw_round_host(dbw_handle* h, const float* X, const double* h_t, const int32_t* h_b,
                    const int32_t* h_batch_idx, const float* G_ext, float lr, float* X_out,
                    uint8_t* h_kept, double* h_T_worker, double* h_T_round, float* h_loss,
-                   void* stream);
+                   int32_t* h_b_out, void* stream);
 
 /*
  * Section 4.1 (threshold rule) and Algorithm 2 (one iteration of the epoch).
@@ -179,6 +181,16 @@ int dbw_status(dbw_handle* h);
 
 /* Spanning links P on the HOST: links[2*(N-1)] receives (u,v) pairs; returns N-1 or an error. */
 int dbw_get_links(const dbw_handle* h, int32_t* links);
+
+/*
+ * Stage timing.  While enabled, every dbw_round / dbw_round_host records CUDA events on the
+ * caller's stream around its stages (0 = gradients, 1 = selection + plan, 2 = mix), up to 4096
+ * rounds.  dbw_profile_read() waits for the recorded events, adds their elapsed times to
+ * ms[3] (HOST), stores the number of rounds in *rounds and clears the record.  Do not enable
+ * it while the stream is being captured into a CUDA graph.
+ */
+int dbw_profile(dbw_handle* h, int enable);
+int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds);
 
 /* Kernels launched by this library since it was loaded (for launch accounting). */
 int64_t dbw_launch_count(void);

@@ -52,13 +52,15 @@ _SIGNATURES = {
     "dbw_mix_in_place_ok": (C.c_int, [_P]),
     "dbw_set_mix_panel": (C.c_int, [_P, C.c_int32]),
     "dbw_round": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P, _P]),
-    "dbw_round_host": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P]),
+    "dbw_round_host": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_update_backups": (C.c_int, [_P, _P, _P, _P, _P]),
     "dbw_reset_backups": (C.c_int, [_P, _P]),
     "dbw_state_export": (C.c_int, [_P, _P, C.POINTER(C.c_size_t), _P]),
     "dbw_state_import": (C.c_int, [_P, _P, C.c_size_t, _P]),
     "dbw_status": (C.c_int, [_P]),
     "dbw_get_links": (C.c_int, [_P, _P]),
+    "dbw_profile": (C.c_int, [_P, C.c_int]),
+    "dbw_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
     "dbw_launch_count": (C.c_int64, []),
     "dbw_last_cuda_error": (C.c_int, []),
 }
@@ -208,10 +210,10 @@ class Dbw:
                                _ptr(T_round), _ptr(loss), _stream()), "dbw_round")
 
     def round_host(self, X, h_t, h_b, lr: float, X_out, h_batch_idx=None, G_ext=None, h_kept=None,
-                   h_T_worker=None, h_T_round=None, h_loss=None):
+                   h_T_worker=None, h_T_round=None, h_loss=None, h_b_out=None):
         _check(lib().dbw_round_host(self._h, _ptr(X), _ptr(h_t), _ptr(h_b), _ptr(h_batch_idx), _ptr(G_ext),
                                     float(lr), _ptr(X_out), _ptr(h_kept), _ptr(h_T_worker), _ptr(h_T_round),
-                                    _ptr(h_loss), _stream()), "dbw_round_host")
+                                    _ptr(h_loss), _ptr(h_b_out), _stream()), "dbw_round_host")
 
     def update_backups(self, t_next, b_out, theta_out=None):
         _check(lib().dbw_update_backups(self._h, _ptr(t_next), _ptr(b_out), _ptr(theta_out), _stream()),
@@ -229,6 +231,16 @@ class Dbw:
 
     def state_import(self, blob: bytes):
         _check(lib().dbw_state_import(self._h, blob, len(blob), _stream()), "dbw_state_import")
+
+    def profile(self, enable: bool):
+        _check(lib().dbw_profile(self._h, int(bool(enable))), "dbw_profile")
+
+    def profile_read(self):
+        """({'grad': ms, 'select': ms, 'mix': ms}, rounds) accumulated since the last read."""
+        ms = (C.c_double * 3)(0.0, 0.0, 0.0)
+        n = C.c_int32(0)
+        _check(lib().dbw_profile_read(self._h, ms, C.byref(n)), "dbw_profile_read")
+        return {"grad": ms[0], "select": ms[1], "mix": ms[2]}, int(n.value)
 
     def status(self) -> int:
         return _check(lib().dbw_status(self._h), "dbw_status")

@@ -110,6 +110,8 @@ int dev_alloc(T** p, size_t n) {
 }
 
 void free_all(dbw_handle* h) {
+    for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+    h->prof_events.clear();
     grad_fp32_free(h);
     grad_bf16_free(h);
     void* ptrs[] = {h->d_rowptr, h->d_col, h->d_links, h->d_covered, h->d_epoch, h->d_status, h->d_waited,
@@ -145,6 +147,7 @@ struct StateBlob {
     // followed by n_links int32 covered flags
 };
 constexpr uint32_t kStateMagic = 0x44425731u;  // "DBW1"
+constexpr int kProfMaxRounds = 4096;
 
 }  // namespace
 
@@ -316,26 +319,67 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
         G = h->d_G;
     }
     if ((rc = check_mix_args(h, X, G, X_out))) return rc;
+    cudaEvent_t* ev = nullptr;
+    if (h->profiling && h->prof_rounds < kProfMaxRounds) {
+        while ((int)h->prof_events.size() < 4 * (h->prof_rounds + 1)) {
+            cudaEvent_t e;
+            DBW_CUDA(cudaEventCreate(&e));
+            h->prof_events.push_back(e);
+        }
+        ev = &h->prof_events[4 * h->prof_rounds++];
+        DBW_CUDA(cudaEventRecord(ev[0], s));
+    }
     if (batch_idx) {
         rc = (h->flags & DBW_GEMM_BF16) ? launch_grad_bf16(h, X, batch_idx, h->d_G, loss, s)
                                         : launch_grad_fp32(h, X, batch_idx, h->d_G, loss, s);
         if (rc) return rc;
     }
+    if (ev) DBW_CUDA(cudaEventRecord(ev[1], s));
     if ((rc = launch_select(h, t, b, kept, T_worker, T_nbr, T_round, true, s))) return rc;
-    return launch_mix(h, X, G, lr, lr_per_worker, X_out, s);
+    if (ev) DBW_CUDA(cudaEventRecord(ev[2], s));
+    rc = launch_mix(h, X, G, lr, lr_per_worker, X_out, s);
+    if (ev) DBW_CUDA(cudaEventRecord(ev[3], s));
+    return rc;
+}
+
+int dbw_profile(dbw_handle* h, int enable) {
+    if (!h) return DBW_ERR_NULL;
+    h->profiling = enable != 0;
+    return DBW_OK;
+}
+
+int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds) {
+    if (!h || !ms || !rounds) return DBW_ERR_NULL;
+    DeviceGuard guard(h->device);
+    for (int r = 0; r < h->prof_rounds; ++r) {
+        cudaEvent_t* ev = &h->prof_events[4 * r];
+        DBW_CUDA(cudaEventSynchronize(ev[3]));
+        for (int st = 0; st < 3; ++st) {
+            float v = 0.f;
+            DBW_CUDA(cudaEventElapsedTime(&v, ev[st], ev[st + 1]));
+            ms[st] += v;
+        }
+    }
+    *rounds = h->prof_rounds;
+    h->prof_rounds = 0;
+    return DBW_OK;
 }
 
 int dbw_round_host(dbw_handle* h, const float* X, const double* h_t, const int32_t* h_b,
                    const int32_t* h_batch_idx, const float* G_ext, float lr, float* X_out, uint8_t* h_kept,
-                   double* h_T_worker, double* h_T_round, float* h_loss, void* stream) {
-    if (!h || !X || !h_t || !h_b || !X_out) return DBW_ERR_NULL;
+                   double* h_T_worker, double* h_T_round, float* h_loss, int32_t* h_b_out, void* stream) {
+    if (!h || !X || !h_t || !X_out) return DBW_ERR_NULL;
     if (!h_batch_idx && !G_ext) return DBW_ERR_NULL;
     DeviceGuard guard(h->device);
     cudaStream_t s = (cudaStream_t)stream;
     int rc;
     if ((rc = ensure_staging(h))) return rc;
     DBW_CUDA(cudaMemcpyAsync(h->s_t, h_t, (size_t)h->N * sizeof(double), cudaMemcpyHostToDevice, s));
-    DBW_CUDA(cudaMemcpyAsync(h->s_b, h_b, (size_t)h->N * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    if (h_b) {
+        DBW_CUDA(cudaMemcpyAsync(h->s_b, h_b, (size_t)h->N * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    } else if ((rc = launch_update_backups(h, h->s_t, h->s_b, nullptr, s))) {
+        return rc;
+    }
     if (h_batch_idx) {
         if (!h->has_model) return DBW_ERR_BAD_MODEL;
         DBW_CUDA(cudaMemcpyAsync(h->s_bidx, h_batch_idx, (size_t)h->N * h->model.batch * sizeof(int32_t),
@@ -347,6 +391,7 @@ int dbw_round_host(dbw_handle* h, const float* X, const double* h_t, const int32
     if (h_kept) DBW_CUDA(cudaMemcpyAsync(h_kept, h->s_kept, (size_t)h->nnz, cudaMemcpyDeviceToHost, s));
     if (h_T_worker) DBW_CUDA(cudaMemcpyAsync(h_T_worker, h->s_Tw, (size_t)h->N * sizeof(double), cudaMemcpyDeviceToHost, s));
     if (h_T_round) DBW_CUDA(cudaMemcpyAsync(h_T_round, h->s_Tr, sizeof(double), cudaMemcpyDeviceToHost, s));
+    if (h_b_out) DBW_CUDA(cudaMemcpyAsync(h_b_out, h->s_b, (size_t)h->N * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     if (h_loss && h_batch_idx) DBW_CUDA(cudaMemcpyAsync(h_loss, h->s_loss, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost, s));
     return DBW_OK;
 }

@@ -88,6 +88,11 @@ struct dbw_handle {
     float* d_G = nullptr;                   // [N][ld] gradient workspace of dbw_round (lazy)
     dbw::BF16State* bf16 = nullptr;
 
+    // stage timing (dbw_profile): events[round][stage boundary 0..3]
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_events;
+    int prof_rounds = 0;
+
     // device staging of dbw_round_host
     double* s_t = nullptr;
     int32_t* s_b = nullptr;
