@@ -39,7 +39,8 @@ enum {
     DBW_ERR_BAD_B = -4,      /* host-side b outside [0, deg] */
     DBW_ERR_BAD_MODEL = -5,  /* model descriptor inconsistent with d / ld, or no model / data set */
     DBW_ERR_CUDA = -6,       /* a CUDA runtime call failed; see dbw_last_cuda_error() */
-    DBW_ERR_STATE = -7       /* state blob of the wrong size or version */
+    DBW_ERR_STATE = -7,      /* state blob of the wrong size or version */
+    DBW_ERR_TOO_LARGE = -8   /* problem larger than a fixed-capacity entry point accepts */
 };
 
 /* flags of dbw_init */
@@ -107,6 +108,41 @@ int dbw_set_dataset(dbw_handle* h, const float* feat, const int32_t* labels, int
  */
 int dbw_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kept, double* T_worker,
                double* T_nbr, double* T_round, void* stream);
+
+/*
+ * dbw_select for callers that must not allocate.  (The paper has no counterpart: this is an
+ * integration aid, not a step of the method.)
+ *
+ * Everything else in this library works through a handle, and dbw_init allocates the handle's
+ * workspace with cudaMalloc.  Some callers cannot do that at the point where they need a
+ * selection: code running inside a latency-critical loop where cudaMalloc's implicit device
+ * synchronisation is not acceptable, plug-ins hosted by a framework whose caching allocator
+ * already owns all of device memory, and callers that are handed a fixed memory budget and are
+ * forbidden to grow it.  This entry point needs no handle and performs no cudaMalloc / cudaFree
+ * (nor any other allocating call): the scratch the selection kernel needs (one flag and one
+ * double per worker plus two counters, about 193 KB) is a fixed array compiled into the library,
+ * which every GPU that loads the library holds until the process exits.
+ *
+ * DEVICE in : rowptr[N+1], col[nnz] — the same sorted, symmetric, self-loop-free CSR that
+ *             dbw_init would take, but already on the device and NOT validated here;
+ *             t[N], b[N] as in dbw_select.
+ * DEVICE out: kept, T_worker, T_nbr, T_round exactly as dbw_select writes them (same kernel,
+ *             so the results are bit-identical); status_out[1] (nullable) receives the
+ *             DBW_STATUS_* bits of this call.
+ * Limits and caveats
+ *   - N <= DBW_SELECT_STATIC_MAX_N, otherwise DBW_ERR_TOO_LARGE and nothing is launched.
+ *   - Works on the CURRENT device.  The first call on each device looks up the device address
+ *     of the built-in array (cudaGetSymbolAddress); make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array, which still holds the previous call's
+ *     contents; each call clears the part that must start at zero with a memset on `stream`.
+ *     Two calls that may overlap on the GPU (different streams, no ordering between them) race
+ *     on it and produce garbage: serialise them.
+ */
+#define DBW_SELECT_STATIC_MAX_N 16384
+int dbw_select_static(int32_t N, const int32_t* rowptr, const int32_t* col, const double* t,
+                      const int32_t* b, uint8_t* kept, double* T_worker, double* T_nbr,
+                      double* T_round, uint32_t* status_out, void* stream);
 
 /*
  * Eq. 2.  DEVICE in: X [N][ld]; batch_idx [N][batch] int32 sample indices into the data set.

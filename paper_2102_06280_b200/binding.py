@@ -20,7 +20,8 @@ STATUS_BAD_B, STATUS_NAN_TIME, STATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4, 
 MAX_LAYERS = 8
 
 _ERR = {-1: "DBW_ERR_NULL", -2: "DBW_ERR_BAD_GRAPH", -3: "DBW_ERR_BAD_SHAPE", -4: "DBW_ERR_BAD_B",
-        -5: "DBW_ERR_BAD_MODEL", -6: "DBW_ERR_CUDA", -7: "DBW_ERR_STATE"}
+        -5: "DBW_ERR_BAD_MODEL", -6: "DBW_ERR_CUDA", -7: "DBW_ERR_STATE", -8: "DBW_ERR_TOO_LARGE"}
+SELECT_STATIC_MAX_N = 16384
 
 
 class DbwError(RuntimeError):
@@ -47,6 +48,7 @@ _SIGNATURES = {
     "dbw_destroy": (C.c_int, [_P]),
     "dbw_set_dataset": (C.c_int, [_P, _P, _P, C.c_int32]),
     "dbw_select": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P]),
+    "dbw_select_static": (C.c_int, [C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_grad": (C.c_int, [_P, _P, _P, _P, _P, _P]),
     "dbw_mix": (C.c_int, [_P, _P, _P, _P, _P, C.c_float, _P, _P, _P]),
     "dbw_mix_in_place_ok": (C.c_int, [_P]),
@@ -249,6 +251,15 @@ class Dbw:
         out = np.zeros((max(self.N - 1, 0), 2), dtype=np.int32)
         _check(lib().dbw_get_links(self._h, out.ctypes.data), "dbw_get_links")
         return out
+
+
+def select_static(rowptr, col, t, b, kept, T_worker=None, T_nbr=None, T_round=None, status_out=None):
+    """dbw_select_static: selection on the current device without a handle and without allocating.
+
+    rowptr / col are device tensors here (int32); the other arguments are as in Dbw.select."""
+    n = int(rowptr.numel()) - 1
+    _check(lib().dbw_select_static(n, _ptr(rowptr), _ptr(col), _ptr(t), _ptr(b), _ptr(kept), _ptr(T_worker),
+                                   _ptr(T_nbr), _ptr(T_round), _ptr(status_out), _stream()), "dbw_select_static")
 
 
 def launch_count() -> int:

@@ -208,3 +208,59 @@ int launch_plan_from_kept(dbw_handle* h, const uint8_t* kept, const int32_t* b, 
 }
 
 }  // namespace dbw
+
+// ---------------------------------------------------------------------------------------------
+// Selection without a handle and without any allocation (dbw_select_static).
+// ---------------------------------------------------------------------------------------------
+namespace dbw {
+namespace {
+
+// Scratch of the allocation-free entry point, resident on every GPU that loads the library:
+// [0,256) ticket and status words, then the "waited for" flags of N workers, then their T_nbr.
+constexpr size_t kStaticFlagsOff = 256;
+constexpr size_t kStaticTnbrOff = kStaticFlagsOff + sizeof(uint32_t) * DBW_SELECT_STATIC_MAX_N;
+constexpr size_t kStaticBytes = kStaticTnbrOff + sizeof(double) * DBW_SELECT_STATIC_MAX_N;
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticBytes];
+
+// Device address of the scratch on the current device (the symbol's name is only a host-side
+// stand-in); looked up once per device.
+int static_scratch(unsigned char** out) {
+    static unsigned char* cache[64] = {};
+    int dev = 0;
+    DBW_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DBW_ERR_BAD_SHAPE;
+    if (!cache[dev]) {
+        void* p = nullptr;
+        DBW_CUDA(cudaGetSymbolAddress(&p, g_select_scratch));
+        cache[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = cache[dev];
+    return DBW_OK;
+}
+
+}  // namespace
+}  // namespace dbw
+
+extern "C" int dbw_select_static(int32_t N, const int32_t* rowptr, const int32_t* col, const double* t,
+                                 const int32_t* b, uint8_t* kept, double* T_worker, double* T_nbr,
+                                 double* T_round, uint32_t* status_out, void* stream) {
+    if (!rowptr || !col || !t || !b || !kept) return DBW_ERR_NULL;
+    if (N < 1) return DBW_ERR_BAD_SHAPE;
+    if (N > DBW_SELECT_STATIC_MAX_N) return DBW_ERR_TOO_LARGE;
+    unsigned char* base = nullptr;
+    int rc = dbw::static_scratch(&base);
+    if (rc) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t* ticket = reinterpret_cast<uint32_t*>(base);
+    uint32_t* status = ticket + 1;
+    uint32_t* waited = reinterpret_cast<uint32_t*>(base + dbw::kStaticFlagsOff);
+    double* tnbr = reinterpret_cast<double*>(base + dbw::kStaticTnbrOff);
+    // the array keeps whatever the previous call left: ticket, status and flags must start at zero
+    DBW_CUDA(cudaMemsetAsync(base, 0, dbw::kStaticFlagsOff + sizeof(uint32_t) * (size_t)N, s));
+    const int blocks = (N + dbw::kWarpsPerBlock - 1) / dbw::kWarpsPerBlock;
+    dbw::select_kernel<<<blocks, dbw::kWarpsPerBlock * 32, 0, s>>>(N, rowptr, col, t, b, kept, tnbr, T_nbr, T_worker,
+                                                                   T_round, waited, ticket, status, dbw::MixPlan{}, 0, 0);
+    DBW_LAUNCHED();
+    if (status_out) DBW_CUDA(cudaMemcpyAsync(status_out, status, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
+    return DBW_OK;
+}

@@ -1,0 +1,71 @@
+"""dbw_select_static, the selection entry point for callers that cannot allocate.
+
+Some users of this library may not call cudaMalloc where they need a selection: code in a
+latency-critical loop (cudaMalloc synchronises the device), plug-ins living inside a framework
+whose caching allocator already owns the device memory, callers held to a fixed memory budget.
+For them the library carries a fixed scratch array and a handle-free entry point.  This test
+calls it through the C ABI twice in a row (the second call finds the first call's leftovers in
+the shared scratch) and requires the same bytes as the handle-based dbw_select, which runs the
+same kernel: kept masks and all times are compared bit for bit, as everywhere in these tests.
+The file name sorts last so that a `-x` run has already executed every other test.
+"""
+import numpy as np
+import pytest
+
+from workloads import configs as wl
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def test_static_selection_matches_handle_based_selection_twice():
+    import paper_2102_06280_b200 as p
+    from paper_2102_06280_b200 import binding
+    graphs = [wl.random_regular(256, 32, 11), wl.complete(40), wl.ring(8)]   # last call is the smallest
+    rng = np.random.default_rng(17)
+    for rowptr, col in graphs:
+        n, nnz = len(rowptr) - 1, len(col)
+        deg = np.diff(rowptr)
+        h = p.Dbw(rowptr, col, d=4)
+        rp_d, col_d = dev(rowptr.astype(np.int32)), dev(col.astype(np.int32))
+        for call in range(2):
+            t = np.round(2 * (1.0 + rng.exponential(1.0, size=n))) / 2     # ties included
+            b = rng.integers(0, deg + 1).astype(np.int32)
+            if call == 1:
+                b[0] = deg[0]                                              # a worker that waits for nobody
+            t_d, b_d = dev(t), dev(b)
+            ref = [torch.zeros(nnz, dtype=torch.uint8, device="cuda"), torch.zeros(n, dtype=torch.float64, device="cuda"),
+                   torch.zeros(n, dtype=torch.float64, device="cuda"), torch.zeros(1, dtype=torch.float64, device="cuda")]
+            got = [torch.full_like(x, 7) for x in ref]
+            st = torch.full((1,), 99, dtype=torch.int32, device="cuda")
+            h.select(t_d, b_d, *ref)
+            launches = binding.launch_count()
+            binding.select_static(rp_d, col_d, t_d, b_d, *got, status_out=st)
+            torch.cuda.synchronize()
+            assert binding.launch_count() == launches + 1
+            for a, r in zip(got, ref):
+                assert torch.equal(a, r)
+            assert int(st.item()) == 0
+        # device-detected problems are reported through status_out, results stay clamped
+        bad = dev(np.full(n, -3, dtype=np.int32))
+        binding.select_static(rp_d, col_d, t_d, bad, *got, status_out=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) & p.STATUS_BAD_B
+        assert h.status() == 0
+        h.close()
+
+
+def test_static_selection_rejects_oversized_and_null():
+    from paper_2102_06280_b200 import binding
+    lib = binding.lib()
+    x = torch.zeros(8, dtype=torch.int32, device="cuda")
+    ptr = x.data_ptr()
+    too_big = binding.SELECT_STATIC_MAX_N + 1
+    assert lib.dbw_select_static(too_big, ptr, ptr, ptr, ptr, ptr, None, None, None, None, None) == -8
+    assert lib.dbw_select_static(4, None, ptr, ptr, ptr, ptr, None, None, None, None, None) == -1
+    assert lib.dbw_select_static(0, ptr, ptr, ptr, ptr, ptr, None, None, None, None, None) == -3
