@@ -1,10 +1,605 @@
-// BF16 tensor-core gradient path (placeholder until the tcgen05 kernels land).
+// Mini-batch stochastic gradient (Eq. 2) with the dense layers on the 5th-generation tensor cores:
+// BF16 operands (activations, and weights cast from the fp32 master rows every round), fp32
+// accumulation in tensor memory, fp32 gradients.  All GEMMs are "both operands K-major":
+//   forward   Z_{l+1} = A_l W_l^T          A-operand A_l      [B][in]    B-operand W_l        [out][in]
+//   dW_l            = dZ_{l+1}^T A_l       A-operand dZ_{l+1}^T [out][B]  B-operand A_l^T      [in][B]
+//   dA_l            = dZ_{l+1} W_l         A-operand dZ_{l+1} [B][out]   B-operand W_l^T      [in][out]
+// so every producer of an activation or of a dZ also writes its transpose.  Tiles are staged by
+// TMA (3-D maps: K, rows, worker; 128-byte swizzle; no multicast) through an mbarrier ring, one
+// elected thread issues tcgen05.mma, and four warps drain the accumulator with tcgen05.ld into the
+// fused epilogues (bias + ReLU + bf16 cast, ReLU mask, or fp32 straight into G).  The last layer
+// (a handful of classes) and the loss run on the CUDA cores from the fp32 master weights.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <vector>
+
 #include "common.cuh"
 
 namespace dbw {
-int grad_bf16_alloc(dbw_handle*) { return DBW_ERR_BAD_MODEL; }
-void grad_bf16_free(dbw_handle*) {}
-int launch_grad_bf16(dbw_handle*, const float*, const int32_t*, float*, float*, cudaStream_t) {
-    return DBW_ERR_BAD_MODEL;
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: after kSpinLimit failed polls the status word is flagged and the caller goes on,
+// so that every role still reaches the end of the kernel and tensor memory is released.
+constexpr uint32_t kSpinLimit = 1u << 24;
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return;
+    atomicOr(status, DBW_STATUS_WAIT_TIMEOUT);
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile staged by TMA with the 128-byte swizzle:
+// rows are 128 bytes (64 bf16) apart, groups of 8 rows 1024 bytes apart (stride byte offset),
+// leading byte offset 16 (unused by this layout), descriptor version 1, layout type 2 = 128B.
+__device__ __forceinline__ uint64_t kmajor_sw128_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// two floats -> packed bf16x2 (low half = first)
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ bool bf16_bits_positive(uint32_t bits16) { return (bits16 & 0x8000u) == 0 && (bits16 & 0x7fffu) != 0; }
+
+// ----------------------------------------------------------------------------- tensor-core GEMM
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3, UMMA_K = 16;
+constexpr int TILE_BYTES = BM * BK * 2;  // 16 KiB per operand tile
+constexpr int GEMM_THREADS = 192;
+constexpr size_t GEMM_SMEM = (size_t)STAGES * 2 * TILE_BYTES + 1024 /*align slack*/ + 128 /*barriers*/;
+// kind::f16, D = f32, A = B = bf16, both K-major, N = 128, M = 128
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+enum { EPI_FWD = 0, EPI_DA = 1, EPI_DW = 2 };
+
+struct TcArgs {
+    int M, N, K, epi;
+    bf16* out;  long long out_z;  int out_pitch;    // [M][N] bf16 (EPI_FWD, EPI_DA)
+    bf16* outT; long long outT_z; int outT_pitch;   // [N][M] bf16, nullable
+    float* outf; long long outf_z; long long outf_pitch;  // [M][N] fp32 (EPI_DW)
+    const float* bias; long long bias_z;            // fp32 [N] (EPI_FWD)
+    const bf16* mask; long long mask_z; int mask_pitch;   // bf16 [M][N]: keep where > 0 (EPI_DA)
+    uint32_t* status;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* tilesA = smem;
+    uint8_t* tilesB = smem + STAGES * TILE_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + 2 * STAGES * TILE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
+    const int num_kb = (g.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                if (kb >= STAGES) mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1, g.status);
+                mbar_expect_tx(&full[s], 2 * TILE_BYTES);
+                tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
+                tma_load_3d(tilesB + s * TILE_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                mbar_wait(&full[s], (kb / STAGES) & 1, g.status);
+                tc_fence_after();
+                const uint64_t da = kmajor_sw128_desc(smem_u32(tilesA + s * TILE_BYTES));
+                const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes further along K inside the swizzle atom
+                    tc_mma_bf16(tmem_base, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
+                                (kb > 0 || k > 0) ? 1u : 0u);
+                tc_commit(&empty[s]);  // frees the stage once these MMAs have read it
+            }
+            tc_commit(acc_full);
+        }
+    } else {
+        // ---- epilogue: warp w owns accumulator lanes 32*(w%4) .. +31, i.e. those output rows ----
+        mbar_wait(acc_full, 0, g.status);
+        tc_fence_after();
+        const int q = warp & 3;
+        const int m = m0 + q * 32 + lane;
+        const bool m_ok = m < g.M;
+        for (int c = 0; c < BN / 32; ++c) {
+            const int nb = n0 + c * 32;
+            if (nb >= g.N) break;  // warp-uniform
+            uint32_t r[32];
+            tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+            if (g.epi == EPI_DW) {
+                if (m_ok) {
+                    float* dst = g.outf + (size_t)z * g.outf_z + (size_t)m * g.outf_pitch + nb;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        if (nb + j < g.N)
+                            *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                              __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                }
+                continue;
+            }
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            if (g.epi == EPI_FWD) {
+                const float* bias = g.bias + (size_t)z * g.bias_z + nb;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + ((nb + j < g.N) ? __ldg(bias + j) : 0.f), 0.f);
+            } else if (m_ok) {  // EPI_DA: ReLU'(z) = [a > 0]
+                const bf16* mk = g.mask + (size_t)z * g.mask_z + (size_t)m * g.mask_pitch + nb;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8)
+                    if (nb + j < g.N) {
+                        const uint4 u = __ldg(reinterpret_cast<const uint4*>(mk + j));
+                        const uint32_t wds[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (!bf16_bits_positive((wds[e >> 1] >> (16 * (e & 1))) & 0xffffu)) v[j + e] = 0.f;
+                    }
+            }
+            uint32_t o[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+            if (m_ok) {
+                bf16* dst = g.out + (size_t)z * g.out_z + (size_t)m * g.out_pitch + nb;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8)
+                    if (nb + j < g.N)
+                        *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[j / 2], o[j / 2 + 1], o[j / 2 + 2], o[j / 2 + 3]);
+                if (g.outT) {
+                    unsigned short* dt = reinterpret_cast<unsigned short*>(g.outT + (size_t)z * g.outT_z + (size_t)nb * g.outT_pitch + m);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nb + j < g.N) dt[(size_t)j * g.outT_pitch] = (unsigned short)((o[j >> 1] >> (16 * (j & 1))) & 0xffffu);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    }
+}
+
+// ----------------------------------------------------------------------------- casts and gathers
+// fp32 [rows][cols] (row pitch src_pitch) -> bf16 [rows][cols] and, if dstT, bf16 [cols][rows].
+// Rows may be indirect (row_idx: mini-batch gather).  32x32 tiles, block (32, 8).
+__global__ void __launch_bounds__(256)
+cast_tile_kernel(int rows, int cols, const float* __restrict__ src, long long src_z, long long src_pitch,
+                 const int32_t* __restrict__ row_idx, int idx_z, int idx_limit, bf16* __restrict__ dst, long long dst_z,
+                 bf16* __restrict__ dstT, long long dstT_z, uint32_t* status) {
+    __shared__ float tile[32][33];
+    const int z = blockIdx.z;
+    const int c = blockIdx.x * 32 + threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = blockIdx.y * 32 + threadIdx.y + 8 * k;
+        float v = 0.f;
+        if (r < rows && c < cols) {
+            long long sr = r;
+            if (row_idx) {
+                int s = row_idx[(size_t)z * idx_z + r];
+                if (s < 0 || s >= idx_limit) {
+                    atomicOr(status, DBW_STATUS_BAD_INDEX);
+                    s = s < 0 ? 0 : idx_limit - 1;
+                }
+                sr = s;
+            }
+            v = __ldg(src + (size_t)z * src_z + sr * src_pitch + c);
+            dst[(size_t)z * dst_z + (size_t)r * cols + c] = __float2bfloat16_rn(v);
+        }
+        tile[threadIdx.y + 8 * k][threadIdx.x] = v;
+    }
+    if (!dstT) return;
+    __syncthreads();
+    const int r2 = blockIdx.y * 32 + threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int c2 = blockIdx.x * 32 + threadIdx.y + 8 * k;
+        if (r2 < rows && c2 < cols) dstT[(size_t)z * dstT_z + (size_t)c2 * rows + r2] = __float2bfloat16_rn(tile[threadIdx.x][threadIdx.y + 8 * k]);
+    }
+}
+
+__global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
+                                     int32_t* __restrict__ ylab) {
+    const int i = blockIdx.x;
+    for (int s = threadIdx.x; s < B; s += blockDim.x) {
+        int src = batch_idx[(size_t)i * B + s];
+        src = src < 0 ? 0 : (src >= S ? S - 1 : src);
+        ylab[(size_t)i * B + s] = labels[(size_t)i * S + src];
+    }
+}
+
+// db[o] = sum over the batch of dZ[.][o], read from the transposed copy dZ^T [out][B]; warp per row.
+__global__ void __launch_bounds__(128)
+bias_grad_t_kernel(int out_dim, int B, const bf16* __restrict__ dzT, long long dzT_z, float* __restrict__ G, long long ld,
+                   long long b_off) {
+    const int i = blockIdx.y;
+    const int o = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (o >= out_dim) return;
+    const bf16* p = dzT + (size_t)i * dzT_z + (size_t)o * B;
+    float s = 0.f;
+    for (int m = lane; m < B; m += 32) s += __bfloat162float(p[m]);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) s += __shfl_xor_sync(0xffffffffu, s, k);
+    if (lane == 0) G[(size_t)i * ld + b_off + o] = s;
+}
+
+// ----------------------------------------------------------------------------- last layer on CUDA cores
+constexpr int kMaxClasses = 32;
+
+// logits = A W^T + b (A bf16 [B][K], W fp32 master [C][K]), then dZ = (softmax - onehot)/B and the
+// per-sample loss.  One warp per sample.
+__global__ void __launch_bounds__(256)
+head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld, long long w_off,
+                    long long b_off, const int32_t* __restrict__ ylab, float* __restrict__ dzL, float* __restrict__ loss_s) {
+    const int i = blockIdx.y;
+    const int s = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (s >= B) return;
+    const bf16* a = A + ((size_t)i * B + s) * K;
+    const float* W = X + (size_t)i * ld + w_off;
+    float z_mine = 0.f;  // lane c ends up holding logit c
+    for (int c = 0; c < C; ++c) {
+        float acc = 0.f;
+        for (int k = lane; k < K; k += 32) acc = fmaf(__bfloat162float(a[k]), __ldg(W + (size_t)c * K + k), acc);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == c) z_mine = acc + X[(size_t)i * ld + b_off + c];
+    }
+    const float zl = lane < C ? z_mine : -INFINITY;
+    float mx = zl;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float e = lane < C ? expf(zl - mx) : 0.f;
+    float sum = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const int y = ylab[(size_t)i * B + s];
+    if (lane < C) dzL[((size_t)i * B + s) * C + lane] = (e / sum - (lane == y ? 1.f : 0.f)) / (float)B;
+    const float zy = __shfl_sync(0xffffffffu, zl, y & 31);
+    if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+}
+
+__global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, float* __restrict__ loss) {
+    const int i = blockIdx.x, lane = threadIdx.x;
+    float s = 0.f;
+    for (int m = lane; m < B; m += 32) s += loss_s[(size_t)i * B + m];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) loss[i] = s / (float)B;
+}
+
+// Last layer backward; thread k of a block owns input feature k:
+//   dW[c][k] = sum_s dZ[s][c] A[s][k],  db[c] = sum_s dZ[s][c],
+//   dZprev[s][k] = [A[s][k] > 0] * sum_c dZ[s][c] W[c][k]   (bf16, plus its transpose [K][B]).
+template <int CP>
+__global__ void __launch_bounds__(128)
+head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld,
+                     long long w_off, long long b_off, const float* __restrict__ dzL, float* __restrict__ G,
+                     bf16* __restrict__ dzP, bf16* __restrict__ dzPT) {
+    extern __shared__ float sdz[];  // [B][CP]
+    const int i = blockIdx.y;
+    for (int e = threadIdx.x; e < B * CP; e += blockDim.x) {
+        const int s = e / CP, c = e % CP;
+        sdz[e] = c < C ? dzL[((size_t)i * B + s) * C + c] : 0.f;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x < C) {
+        float t = 0.f;
+        for (int s = 0; s < B; ++s) t += sdz[s * CP + threadIdx.x];
+        G[(size_t)i * ld + b_off + threadIdx.x] = t;
+    }
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    float w[CP], dw[CP];
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+        w[c] = c < C ? X[(size_t)i * ld + w_off + (size_t)c * K + k] : 0.f;
+        dw[c] = 0.f;
+    }
+    const bf16* a = A + (size_t)i * B * K + k;
+    for (int s0 = 0; s0 < B; s0 += 8) {  // B % 8 == 0
+        float dav[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int s = s0 + u;
+            const float av = __bfloat162float(a[(size_t)s * K]);
+            float da = 0.f;
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                const float dz = sdz[s * CP + c];
+                dw[c] = fmaf(dz, av, dw[c]);
+                da = fmaf(dz, w[c], da);
+            }
+            dav[u] = av > 0.f ? da : 0.f;
+            if (dzP) dzP[((size_t)i * B + s) * K + k] = __float2bfloat16_rn(dav[u]);
+        }
+        if (dzPT)
+            *reinterpret_cast<uint4*>(dzPT + ((size_t)i * K + k) * B + s0) =
+                make_uint4(pack_bf16x2(dav[0], dav[1]), pack_bf16x2(dav[2], dav[3]), pack_bf16x2(dav[4], dav[5]),
+                           pack_bf16x2(dav[6], dav[7]));
+    }
+#pragma unroll
+    for (int c = 0; c < CP; ++c)
+        if (c < C) G[(size_t)i * ld + w_off + (size_t)c * K + k] = dw[c];
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// K-major operand [workers][rows][K] bf16, dense: box = 64 (K) x 128 (rows) x 1, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)workers};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * 2 * (cuuint64_t)rows};
+    cuuint32_t box[3] = {BK, BM, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct BF16State {
+    bf16* A[DBW_MAX_LAYERS] = {};    // A_l   [N][B][dims[l]],  l = 0..L-1
+    bf16* AT[DBW_MAX_LAYERS] = {};   // A_l^T [N][dims[l]][B],  l = 0..L-2
+    bf16* Wh[DBW_MAX_LAYERS] = {};   // W_l   [N][out][in],     l = 0..L-2
+    bf16* WhT[DBW_MAX_LAYERS] = {};  // W_l^T [N][in][out],     l = 1..L-2
+    bf16* dZ[DBW_MAX_LAYERS] = {};   // dZ_l  [N][B][dims[l]],  l = 1..L-1
+    bf16* dZT[DBW_MAX_LAYERS] = {};  // dZ_l^T
+    float* dzL = nullptr;            // [N][B][C]
+    float* loss_s = nullptr;         // [N][B]
+    int32_t* ylab = nullptr;         // [N][B]
+    CUtensorMap fwdA[DBW_MAX_LAYERS], fwdB[DBW_MAX_LAYERS], dwA[DBW_MAX_LAYERS], dwB[DBW_MAX_LAYERS],
+        daA[DBW_MAX_LAYERS], daB[DBW_MAX_LAYERS];
+    std::vector<void*> owned;
+};
+
+namespace {
+template <typename T>
+bool balloc(BF16State* st, T** p, size_t n) {
+    if (!cuda_ok(cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T)))) return false;
+    st->owned.push_back(*p);
+    return true;
+}
+
+int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
+    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, workers);
+    gemm_tc_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(a, b, g);
+    DBW_LAUNCHED();
+    return DBW_OK;
+}
+}  // namespace
+
+int grad_bf16_alloc(dbw_handle* h) {
+    const dbw_model_desc& m = h->model;
+    const int L = m.n_layers, B = m.batch, N = h->N;
+    // TMA needs 16-byte row pitches, the transposed stores 16-byte groups of samples
+    if (B % 8) return DBW_ERR_BAD_MODEL;
+    for (int l = 0; l < L; ++l)
+        if (m.dims[l] % 8) return DBW_ERR_BAD_MODEL;
+    if (m.dims[L] > kMaxClasses) return DBW_ERR_BAD_MODEL;
+    if ((size_t)B * (m.dims[L] <= 16 ? 16 : 32) * 4 > 200 * 1024) return DBW_ERR_BAD_MODEL;
+    BF16State* st = new (std::nothrow) BF16State();
+    if (!st) return DBW_ERR_CUDA;
+    h->bf16 = st;
+    bool ok = true;
+    const size_t NB = (size_t)N * B;
+    for (int l = 0; l < L && ok; ++l) {
+        ok = ok && balloc(st, &st->A[l], NB * m.dims[l]);
+        if (l <= L - 2) {
+            ok = ok && balloc(st, &st->AT[l], NB * m.dims[l]);
+            ok = ok && balloc(st, &st->Wh[l], (size_t)N * m.dims[l] * m.dims[l + 1]);
+            if (l >= 1) ok = ok && balloc(st, &st->WhT[l], (size_t)N * m.dims[l] * m.dims[l + 1]);
+        }
+        if (l >= 1) {
+            ok = ok && balloc(st, &st->dZ[l], NB * m.dims[l]);
+            ok = ok && balloc(st, &st->dZT[l], NB * m.dims[l]);
+        }
+    }
+    ok = ok && balloc(st, &st->dzL, NB * m.dims[L]) && balloc(st, &st->loss_s, NB) && balloc(st, &st->ylab, NB);
+    if (!ok) return DBW_ERR_CUDA;
+    for (int l = 0; l <= L - 2; ++l) {
+        ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
+        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N);
+        ok = ok && make_operand_map(&st->dwA[l], st->dZT[l + 1], B, m.dims[l + 1], N);
+        ok = ok && make_operand_map(&st->dwB[l], st->AT[l], B, m.dims[l], N);
+        if (l >= 1) {
+            ok = ok && make_operand_map(&st->daA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
+            ok = ok && make_operand_map(&st->daB[l], st->WhT[l], m.dims[l + 1], m.dims[l], N);
+        }
+    }
+    if (!ok) return DBW_ERR_CUDA;
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
+    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    return DBW_OK;
+}
+
+void grad_bf16_free(dbw_handle* h) {
+    if (!h->bf16) return;
+    for (void* p : h->bf16->owned) cudaFree(p);
+    delete h->bf16;
+    h->bf16 = nullptr;
+}
+
+int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss, cudaStream_t s) {
+    const dbw_model_desc& m = h->model;
+    BF16State* st = h->bf16;
+    const int L = m.n_layers, B = m.batch, N = h->N, C = m.dims[L];
+    int rc;
+    // bf16 copies of the weights of the tensor-core layers (and their transposes for dA)
+    for (int l = 0; l <= L - 2; ++l) {
+        const int in = m.dims[l], out = m.dims[l + 1];
+        cast_tile_kernel<<<dim3((in + 31) / 32, (out + 31) / 32, N), dim3(32, 8), 0, s>>>(
+            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], (long long)in * out, l >= 1 ? st->WhT[l] : nullptr,
+            (long long)in * out, h->d_status);
+        DBW_LAUNCHED();
+    }
+    // mini-batch gather: A_0 (and A_0^T when a tensor-core layer consumes it)
+    cast_tile_kernel<<<dim3((m.dims[0] + 31) / 32, (B + 31) / 32, N), dim3(32, 8), 0, s>>>(
+        B, m.dims[0], h->feat, (long long)h->S * m.dims[0], m.dims[0], batch_idx, B, h->S, st->A[0], (long long)B * m.dims[0],
+        L >= 2 ? st->AT[0] : nullptr, (long long)B * m.dims[0], h->d_status);
+    DBW_LAUNCHED();
+    gather_labels_kernel<<<N, 128, 0, s>>>(B, h->S, h->labels, batch_idx, st->ylab);
+    DBW_LAUNCHED();
+    // forward through the tensor-core layers
+    for (int l = 0; l <= L - 2; ++l) {
+        TcArgs g{};
+        g.M = B; g.N = m.dims[l + 1]; g.K = m.dims[l]; g.epi = EPI_FWD;
+        g.out = st->A[l + 1]; g.out_z = (long long)B * g.N; g.out_pitch = g.N;
+        g.outT = (l + 1 <= L - 2) ? st->AT[l + 1] : nullptr; g.outT_z = (long long)B * g.N; g.outT_pitch = B;
+        g.bias = X + m.b_off[l]; g.bias_z = h->ld;
+        g.status = h->d_status;
+        if ((rc = run_tc(st->fwdA[l], st->fwdB[l], g, N, s))) return rc;
+    }
+    // last layer, loss, and its backward
+    const int K = m.dims[L - 1];
+    head_forward_kernel<<<dim3((B + 7) / 8, N), 256, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1],
+                                                             st->ylab, st->dzL, st->loss_s);
+    DBW_LAUNCHED();
+    if (loss) {
+        loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
+        DBW_LAUNCHED();
+    }
+    bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
+    bf16* dzPT = L >= 2 ? st->dZT[L - 1] : nullptr;
+    if (C <= 16)
+        head_backward_kernel<16><<<dim3((K + 127) / 128, N), 128, (size_t)B * 16 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
+    else
+        head_backward_kernel<32><<<dim3((K + 127) / 128, N), 128, (size_t)B * 32 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
+    DBW_LAUNCHED();
+    // backward through the tensor-core layers
+    for (int l = L - 2; l >= 0; --l) {
+        const int in = m.dims[l], out = m.dims[l + 1];
+        TcArgs w{};
+        w.M = out; w.N = in; w.K = B; w.epi = EPI_DW;
+        w.outf = G + m.w_off[l]; w.outf_z = h->ld; w.outf_pitch = in;
+        w.status = h->d_status;
+        if ((rc = run_tc(st->dwA[l], st->dwB[l], w, N, s))) return rc;
+        bias_grad_t_kernel<<<dim3((out + 3) / 4, N), 128, 0, s>>>(out, B, st->dZT[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
+        DBW_LAUNCHED();
+        if (l >= 1) {
+            TcArgs a{};
+            a.M = B; a.N = in; a.K = out; a.epi = EPI_DA;
+            a.out = st->dZ[l]; a.out_z = (long long)B * in; a.out_pitch = in;
+            a.outT = st->dZT[l]; a.outT_z = (long long)B * in; a.outT_pitch = B;
+            a.mask = st->A[l]; a.mask_z = (long long)B * in; a.mask_pitch = in;
+            a.status = h->d_status;
+            if ((rc = run_tc(st->daA[l], st->daB[l], a, N, s))) return rc;
+        }
+    }
+    return DBW_OK;
+}
+
 }  // namespace dbw
