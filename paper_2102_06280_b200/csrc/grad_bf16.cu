@@ -194,14 +194,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t r[32];
             tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
             if (g.epi == EPI_DW) {
-                if (m_ok) {
-                    float* dst = g.outf + (size_t)z * g.outf_z + (size_t)m * g.outf_pitch + nb;
+                // Each lane holds one row of a 32 x 32 fp32 block.  It goes through shared memory (the
+                // drained pipeline stages; rows 36 words apart keep both 128-bit phases conflict-free)
+                // so that a warp stores four full 128-byte lines per instruction.
+                float* stg = reinterpret_cast<float*>(smem) + q * (32 * 36);
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4)
-                        if (nb + j < g.N)
-                            *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                              __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<uint4*>(stg + lane * 36 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                __syncwarp();
+                const int f4 = lane & 7;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int row = 4 * i + (lane >> 3);
+                    const int mm = m0 + q * 32 + row;
+                    const float4 val = *reinterpret_cast<const float4*>(stg + row * 36 + 4 * f4);
+                    if (mm < g.M && nb + 4 * f4 < g.N)
+                        *reinterpret_cast<float4*>(g.outf + (size_t)z * g.outf_z + (size_t)mm * g.outf_pitch + nb + 4 * f4) = val;
                 }
+                __syncwarp();
                 continue;
             }
             float v[32];
@@ -251,41 +261,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // ----------------------------------------------------------------------------- casts and gathers
 // fp32 [rows][cols] (row pitch src_pitch) -> bf16 [rows][cols] and, if dstT, bf16 [cols][rows].
-// Rows may be indirect (row_idx: mini-batch gather).  32x32 tiles, block (32, 8).
+// Rows may be indirect (row_idx: mini-batch gather).  cols % 8 == 0 and rows % 8 == 0.
+// A block of 256 threads handles a 64 x 64 tile: every thread loads 16 consecutive floats of one
+// row (four 128-bit loads), stores them as 16 bf16 (two 128-bit stores), and for the transpose the
+// tile passes through shared memory so that the transposed rows leave as 128-bit stores too.
+__device__ __forceinline__ uint4 pack8(const float* v) {
+    return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+}
+
 __global__ void __launch_bounds__(256)
 cast_tile_kernel(int rows, int cols, const float* __restrict__ src, long long src_z, long long src_pitch,
                  const int32_t* __restrict__ row_idx, int idx_z, int idx_limit, bf16* __restrict__ dst, long long dst_z,
                  bf16* __restrict__ dstT, long long dstT_z, uint32_t* status) {
-    __shared__ float tile[32][33];
+    __shared__ float tile[64][65];
     const int z = blockIdx.z;
-    const int c = blockIdx.x * 32 + threadIdx.x;
+    const int t = threadIdx.x;
+    const int r = blockIdx.y * 64 + (t >> 2);
+    const int c0 = blockIdx.x * 64 + (t & 3) * 16;
+    float v[16];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int r = blockIdx.y * 32 + threadIdx.y + 8 * k;
-        float v = 0.f;
-        if (r < rows && c < cols) {
-            long long sr = r;
-            if (row_idx) {
-                int s = row_idx[(size_t)z * idx_z + r];
-                if (s < 0 || s >= idx_limit) {
-                    atomicOr(status, DBW_STATUS_BAD_INDEX);
-                    s = s < 0 ? 0 : idx_limit - 1;
-                }
-                sr = s;
+    for (int e = 0; e < 16; ++e) v[e] = 0.f;
+    if (r < rows) {
+        long long sr = r;
+        if (row_idx) {
+            int s = row_idx[(size_t)z * idx_z + r];
+            if (s < 0 || s >= idx_limit) {
+                atomicOr(status, DBW_STATUS_BAD_INDEX);
+                s = s < 0 ? 0 : idx_limit - 1;
             }
-            v = __ldg(src + (size_t)z * src_z + sr * src_pitch + c);
-            dst[(size_t)z * dst_z + (size_t)r * cols + c] = __float2bfloat16_rn(v);
+            sr = s;
         }
-        tile[threadIdx.y + 8 * k][threadIdx.x] = v;
+        const float* p = src + (size_t)z * src_z + sr * src_pitch + c0;
+        bf16* d = dst + (size_t)z * dst_z + (size_t)r * cols + c0;
+#pragma unroll
+        for (int e = 0; e < 16; e += 4)
+            if (c0 + e < cols) {
+                const float4 f = __ldg(reinterpret_cast<const float4*>(p + e));
+                v[e] = f.x; v[e + 1] = f.y; v[e + 2] = f.z; v[e + 3] = f.w;
+            }
+        if (c0 < cols) *reinterpret_cast<uint4*>(d) = pack8(v);
+        if (c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
     }
     if (!dstT) return;
-    __syncthreads();
-    const int r2 = blockIdx.y * 32 + threadIdx.x;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int c2 = blockIdx.x * 32 + threadIdx.y + 8 * k;
-        if (r2 < rows && c2 < cols) dstT[(size_t)z * dstT_z + (size_t)c2 * rows + r2] = __float2bfloat16_rn(tile[threadIdx.x][threadIdx.y + 8 * k]);
-    }
+    for (int e = 0; e < 16; ++e) tile[t >> 2][(t & 3) * 16 + e] = v[e];
+    __syncthreads();
+    const int c = blockIdx.x * 64 + (t >> 2);
+    const int r0 = blockIdx.y * 64 + (t & 3) * 16;
+    if (c >= cols) return;
+    float w[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) w[e] = tile[(t & 3) * 16 + e][t >> 2];
+    bf16* d = dstT + (size_t)z * dstT_z + (size_t)c * rows + r0;
+    if (r0 < rows) *reinterpret_cast<uint4*>(d) = pack8(w);
+    if (r0 + 8 < rows) *reinterpret_cast<uint4*>(d + 8) = pack8(w + 8);
 }
 
 __global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
@@ -539,13 +568,13 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // bf16 copies of the weights of the tensor-core layers (and their transposes for dA)
     for (int l = 0; l <= L - 2; ++l) {
         const int in = m.dims[l], out = m.dims[l + 1];
-        cast_tile_kernel<<<dim3((in + 31) / 32, (out + 31) / 32, N), dim3(32, 8), 0, s>>>(
+        cast_tile_kernel<<<dim3((in + 63) / 64, (out + 63) / 64, N), 256, 0, s>>>(
             out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], (long long)in * out, l >= 1 ? st->WhT[l] : nullptr,
             (long long)in * out, h->d_status);
         DBW_LAUNCHED();
     }
     // mini-batch gather: A_0 (and A_0^T when a tensor-core layer consumes it)
-    cast_tile_kernel<<<dim3((m.dims[0] + 31) / 32, (B + 31) / 32, N), dim3(32, 8), 0, s>>>(
+    cast_tile_kernel<<<dim3((m.dims[0] + 63) / 64, (B + 63) / 64, N), 256, 0, s>>>(
         B, m.dims[0], h->feat, (long long)h->S * m.dims[0], m.dims[0], batch_idx, B, h->S, st->A[0], (long long)B * m.dims[0],
         L >= 2 ? st->AT[0] : nullptr, (long long)B * m.dims[0], h->d_status);
     DBW_LAUNCHED();
