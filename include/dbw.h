@@ -166,6 +166,7 @@ int dbw_mix(dbw_handle* h, const float* X, const float* G, const uint8_t* kept, 
 int dbw_mix_in_place_ok(const dbw_handle* h);
 /* Expert knob: columns per shared-memory panel of the mix kernel: 0 = automatic, 16 / 32 / 64 /
  * 128 = fixed (falls back to the direct kernel when N * cols * 4 bytes exceed shared memory),
+ * 1 = the tensor-memory staged kernel wherever it applies (uniform weights, 64 <= N <= 1024),
  * -1 = always the direct (L2 re-read, out-of-place only) kernel. */
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols);
 

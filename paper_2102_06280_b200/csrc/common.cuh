@@ -115,6 +115,11 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
                cudaStream_t s);
 bool mix_panel_fits(const dbw_handle* h);
 
+// mix_staged.cu
+bool mix_staged_usable(const dbw_handle* h);
+int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+                      cudaStream_t s);
+
 // dtur.cu
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);
 

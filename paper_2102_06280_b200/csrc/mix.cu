@@ -116,6 +116,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
 
 int auto_group_size(const dbw_handle* h) {
     if (h->mix_panel_cols < 0) return 0;  // direct kernel forced
+    if (h->mix_panel_cols == 1) return 0; // staged kernel forced (handled by the caller)
     if (h->mix_panel_cols) return ((size_t)h->N * h->mix_panel_cols * 4 <= (size_t)h->smem_optin) ? h->mix_panel_cols / 4 : 0;
     // widest panel whose staging buffer still lets two CTAs share an SM
     const size_t budget = (size_t)(h->smem_optin) / 2 - 1024;
@@ -148,10 +149,19 @@ int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const 
 
 }  // namespace
 
-bool mix_panel_fits(const dbw_handle* h) { return auto_group_size(h) != 0; }
+// The tensor-memory staged kernel takes over when it applies and the plain panel kernel could not
+// keep a 32-column (128-byte segment) panel with two CTAs per SM.
+static bool use_staged(const dbw_handle* h) {
+    if (!mix_staged_usable(h)) return false;
+    if (h->mix_panel_cols == 1) return true;
+    return h->mix_panel_cols == 0 && auto_group_size(h) < 8;
+}
+
+bool mix_panel_fits(const dbw_handle* h) { return use_staged(h) || auto_group_size(h) != 0; }
 
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s) {
+    if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, s);
     switch (auto_group_size(h)) {
         case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, s);
         case 16: return launch_panel<16>(h, X, G, lr, lr_pw, X_out, s);

@@ -1,0 +1,260 @@
+// Mix kernel for many workers and many terms per output (uniform weights): one persistent CTA per
+// SM, warp-specialised, with the NEXT column panel prefetched into tensor memory.
+//
+// With N of the order of 1000 a 32-column panel of all rows (N x 128 B) plus the neighbour lists
+// fill shared memory, so there is no room for a second panel buffer, and with about 30 terms per
+// output the gather out of shared memory takes longer than the HBM stream.  To overlap the two,
+// eight producer warps stream the next panel of X and G from HBM (128-bit loads, x - lr*g formed
+// in registers) and park it in the SM's tensor memory with tcgen05.st, while sixteen consumer warps
+// gather the current panel out of shared memory.  When both are done the producers move the parked
+// panel from tensor memory into shared memory (tcgen05.ld + 128-bit shared stores) and the roles
+// repeat.  The neighbour lists (16-bit indices, built once per launch from the mixing plan) stay in
+// shared memory for the whole launch.  HBM traffic is the algorithmic 12 bytes per element; a panel
+// is fully staged before any of it is written and panels are disjoint, so X' may overwrite X.
+#include "common.cuh"
+
+namespace dbw {
+
+namespace {
+
+constexpr int kProdWarps = 8, kConsWarps = 16;
+constexpr int kThreads = (kProdWarps + kConsWarps) * 32;  // 768
+constexpr int kTmemCols = 256;                            // 128 lanes x 256 columns x 4 B = one 1024 x 32 panel
+constexpr int kMaxN = 1024;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float4 (&v)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "f"(v[0].x), "f"(v[0].y), "f"(v[0].z), "f"(v[0].w), "f"(v[1].x), "f"(v[1].y), "f"(v[1].z), "f"(v[1].w),
+        "f"(v[2].x), "f"(v[2].y), "f"(v[2].z), "f"(v[2].w), "f"(v[3].x), "f"(v[3].y), "f"(v[3].z), "f"(v[3].w), "f"(v[4].x),
+        "f"(v[4].y), "f"(v[4].z), "f"(v[4].w), "f"(v[5].x), "f"(v[5].y), "f"(v[5].z), "f"(v[5].w), "f"(v[6].x), "f"(v[6].y),
+        "f"(v[6].z), "f"(v[6].w), "f"(v[7].x), "f"(v[7].y), "f"(v[7].z), "f"(v[7].w)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float4 (&v)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=f"(v[0].x), "=f"(v[0].y), "=f"(v[0].z), "=f"(v[0].w), "=f"(v[1].x), "=f"(v[1].y), "=f"(v[1].z), "=f"(v[1].w),
+          "=f"(v[2].x), "=f"(v[2].y), "=f"(v[2].z), "=f"(v[2].w), "=f"(v[3].x), "=f"(v[3].y), "=f"(v[3].z), "=f"(v[3].w),
+          "=f"(v[4].x), "=f"(v[4].y), "=f"(v[4].z), "=f"(v[4].w), "=f"(v[5].x), "=f"(v[5].y), "=f"(v[5].z), "=f"(v[5].w),
+          "=f"(v[6].x), "=f"(v[6].y), "=f"(v[6].z), "=f"(v[6].w), "=f"(v[7].x), "=f"(v[7].y), "=f"(v[7].z), "=f"(v[7].w)
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void add4(float4& a, const float4 v) {
+    a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+}
+
+struct StagedArgs {
+    int N, n_panels, mix_then_correct, plan_row;  // plan_row: 16-bit entries per neighbour-list row (multiple of 8)
+    long long ld;
+    const float* X;
+    const float* G;
+    float lr;
+    const float* lr_pw;
+    float* Xout;
+    MixPlan plan;
+};
+
+// Shared memory: panel float4 [N + 1][8] (row N is all zero: the target of list padding), then the
+// neighbour lists uint16 [N][plan_row + 8] (the 16-byte skew keeps four consecutive rows in distinct
+// banks), then the per-row scale float [N], then the list lengths in blocks of 8, uint8 [N].
+__global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
+    extern __shared__ float4 smem4[];
+    float4* panel = smem4;
+    const int N = a.N;
+    const int prow = a.plan_row + 8;  // uint16 per list row
+    uint16_t* lists = reinterpret_cast<uint16_t*>(panel + (size_t)(N + 1) * 8);
+    float* scale = reinterpret_cast<float*>(lists + (size_t)N * prow);
+    uint8_t* nblk = reinterpret_cast<uint8_t*>(scale + N);
+    __shared__ uint32_t tmem_slot;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // neighbour lists, scales and the zero row: once per launch
+    for (int e = tid; e < N * (prow / 8); e += kThreads) {
+        const int i = e / (prow / 8), k0 = (e % (prow / 8)) * 8;
+        const int cnt = a.plan.cnt[i];
+        uint32_t w[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const int k = k0 + 2 * h;
+            const uint32_t lo = k < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + k] : (uint32_t)N;
+            const uint32_t hi = k + 1 < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + k + 1] : (uint32_t)N;
+            w[h] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(lists + (size_t)i * prow + k0) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    for (int i = tid; i < N; i += kThreads) {
+        scale[i] = a.plan.w_self[i];
+        nblk[i] = (uint8_t)((a.plan.cnt[i] + 7) / 8);
+    }
+    if (tid < 8) panel[(size_t)N * 8 + tid] = make_float4(0.f, 0.f, 0.f, 0.f);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+
+    const int n_its = (N + 31) / 32;  // a producer warp stages 4 rows per iteration, the eight warps 32
+    const bool producer = warp < kProdWarps;
+    // producer coordinates: row (within an iteration) and 16-byte slot of the 128-byte row segment
+    const int p_row = warp * 4 + (lane >> 3), slot = lane & 7;
+    const uint32_t p_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+    // consumer coordinates: 64 groups of 8 lanes, each group owns rows grp, grp + 64, ...
+    const int grp = (warp - kProdWarps) * 4 + (lane >> 3);
+
+    auto stage = [&](int pn) {  // HBM -> registers -> tensor memory
+        const long long c = (long long)pn * 32 + 4 * slot;
+        const bool c_ok = c < a.ld;
+        for (int bt = 0; bt < n_its; bt += 8) {
+            float4 x[8], g[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int r = (bt + u) * 32 + p_row;
+                const bool ok = c_ok && r < N;
+                x[u] = ok ? ldg4(a.X + (size_t)r * a.ld + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (!a.mix_then_correct) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int r = (bt + u) * 32 + p_row;
+                    const bool ok = c_ok && r < N;
+                    g[u] = ok ? ldg4(a.G + (size_t)r * a.ld + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int r = (bt + u) * 32 + p_row;
+                    const float nlr = -((a.lr_pw && r < N) ? a.lr_pw[r] : a.lr);
+                    x[u].x = fmaf(nlr, g[u].x, x[u].x);
+                    x[u].y = fmaf(nlr, g[u].y, x[u].y);
+                    x[u].z = fmaf(nlr, g[u].z, x[u].z);
+                    x[u].w = fmaf(nlr, g[u].w, x[u].w);
+                }
+            }
+            tmem_st32(p_taddr + (uint32_t)(4 * bt), x);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    };
+    auto unpark = [&]() {  // tensor memory -> shared-memory panel
+        for (int bt = 0; bt < n_its; bt += 8) {
+            float4 x[8];
+            tmem_ld32(p_taddr + (uint32_t)(4 * bt), x);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int r = (bt + u) * 32 + p_row;
+                if (r < N) panel[(size_t)r * 8 + slot] = x[u];
+            }
+        }
+    };
+    auto gather = [&](int pn) {  // every output row of the panel out of shared memory
+        const long long c = (long long)pn * 32 + 4 * slot;
+        for (int i = grp; i < N; i += kConsWarps * 4) {
+            float4 acc = panel[(size_t)i * 8 + slot];
+            const uint4* lp = reinterpret_cast<const uint4*>(lists + (size_t)i * prow);
+            const int nb = nblk[i];
+            for (int kb = 0; kb < nb; ++kb) {
+                const uint4 u = lp[kb];
+                const float4 v0 = panel[(size_t)(u.x & 0xffffu) * 8 + slot], v1 = panel[(size_t)(u.x >> 16) * 8 + slot];
+                const float4 v2 = panel[(size_t)(u.y & 0xffffu) * 8 + slot], v3 = panel[(size_t)(u.y >> 16) * 8 + slot];
+                const float4 v4 = panel[(size_t)(u.z & 0xffffu) * 8 + slot], v5 = panel[(size_t)(u.z >> 16) * 8 + slot];
+                const float4 v6 = panel[(size_t)(u.w & 0xffffu) * 8 + slot], v7 = panel[(size_t)(u.w >> 16) * 8 + slot];
+                add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
+                add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
+            }
+            const float w = scale[i];
+            acc.x *= w; acc.y *= w; acc.z *= w; acc.w *= w;
+            if (c < a.ld) {
+                if (a.mix_then_correct) {
+                    const float4 gi = ldg4(a.G + (size_t)i * a.ld + c);
+                    const float nlr = -(a.lr_pw ? a.lr_pw[i] : a.lr);
+                    acc.x = fmaf(nlr, gi.x, acc.x); acc.y = fmaf(nlr, gi.y, acc.y);
+                    acc.z = fmaf(nlr, gi.z, acc.z); acc.w = fmaf(nlr, gi.w, acc.w);
+                }
+                *reinterpret_cast<float4*>(a.Xout + (size_t)i * a.ld + c) = acc;
+            }
+        }
+    };
+
+    int pn = blockIdx.x;
+    if (pn < a.n_panels) {
+        if (producer) {
+            stage(pn);
+            unpark();
+        }
+        __syncthreads();
+        while (true) {
+            const int next = pn + gridDim.x;
+            const bool more = next < a.n_panels;
+            if (producer) {
+                if (more) stage(next);
+            } else {
+                gather(pn);
+            }
+            __syncthreads();  // panel pn consumed, panel `next` parked
+            if (!more) break;
+            if (producer) unpark();
+            __syncthreads();  // panel `next` in shared memory
+            pn = next;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+size_t staged_smem(const dbw_handle* h, int plan_row) {
+    const size_t N = (size_t)h->N;
+    return (N + 1) * 128 + N * (size_t)(plan_row + 8) * 2 + N * 4 + ((N + 15) / 16) * 16;
+}
+
+}  // namespace
+
+// Usable when the weights are uniform (one scale per row, so a list entry is a bare 16-bit index),
+// every worker's panel row fits the tensor-memory staging area, and the shared memory holds panel
+// and lists.
+bool mix_staged_usable(const dbw_handle* h) {
+    if (!(h->flags & DBW_WEIGHT_UNIFORM)) return false;
+    if (h->N > kMaxN || h->N < 64) return false;
+    const int plan_row = (h->maxdeg + 7) / 8 * 8;
+    if (plan_row > 248) return false;
+    return staged_smem(h, plan_row) + 256 <= (size_t)h->smem_optin;
+}
+
+int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+                      cudaStream_t s) {
+    StagedArgs a{};
+    a.N = h->N;
+    a.ld = h->ld;
+    a.n_panels = (int)((h->ld + 31) / 32);
+    a.mix_then_correct = (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0;
+    a.plan_row = (h->maxdeg + 7) / 8 * 8;
+    a.X = X; a.G = G; a.lr = lr; a.lr_pw = lr_pw; a.Xout = X_out; a.plan = h->plan;
+    const size_t smem = staged_smem(h, a.plan_row);
+    static bool configured[64] = {};
+    if (!configured[h->device & 63]) {
+        DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
+        configured[h->device & 63] = true;
+    }
+    const int grid = a.n_panels < h->sm_count ? a.n_panels : h->sm_count;
+    mix_staged_kernel<<<grid, kThreads, smem, s>>>(a);
+    DBW_LAUNCHED();
+    return DBW_OK;
+}
+
+}  // namespace dbw
