@@ -338,7 +338,12 @@ def run_ours(args):
         build.build()
     if dist is not None:
         dist.barrier()
-    job = Job(args.config, device=local)
+    overrides = {}
+    if args.samples:
+        overrides["samples"] = args.samples
+    if args.width:
+        overrides["d"] = args.width
+    job = Job(args.config, device=local, **overrides)
     w = job.w
     for _ in range(args.warmup):
         job.step()
@@ -405,6 +410,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU oracle work per sampled step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--samples", type=int, default=0, help="profiling aid: samples per worker instead of the config's")
+    ap.add_argument("--width", type=int, default=0, help="profiling aid: columns d of the mix-only config instead of 2^20")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
