@@ -33,6 +33,10 @@ from workloads import configs as wl  # noqa: E402
 METRIC = "simulated worker-rounds/sec"
 UNIT = "worker-rounds/s"
 DEFAULT_CONFIG = 4
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix kernel, from the ncu captures
+# summarised under profiles/ (small case scaled by the columns processed); None = not captured for
+# this workload or the kernel changed since.
+MIX_TRAFFIC_BYTES = {4: (537.3e6 + 219.3e6) * 16}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -301,6 +305,21 @@ def run_reference(args):
 # the GPU arm
 # ------------------------------------------------------------------------------------------
 
+def max_over_ranks(ms, dist, device="cuda"):
+    """Slowest rank's time (every rank gets it); `dist` is torch.distributed or None."""
+    if dist is None:
+        return float(ms)
+    import torch
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def aggregate_value(units_per_rank_step, steps, ms_max, world):
+    """Whole-job throughput of `world` replicas: all units processed / slowest rank's time."""
+    return world * units_per_rank_step * steps / (ms_max * 1e-3)
+
+
 def timed_loop(job, steps, fn, dist):
     import torch
     if dist is not None:
@@ -314,12 +333,7 @@ def timed_loop(job, steps, fn, dist):
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tt = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
-    return ms
+    return max_over_ranks(e0.elapsed_time(e1), dist)
 
 
 def run_ours(args):
@@ -370,14 +384,16 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     peaks, peak_kind = measured_peaks()
-    value = world * w.N * args.steps / (ms * 1e-3)
-    e2e = world * w.N * args.steps / (ms_e2e * 1e-3)
+    value = aggregate_value(w.N, args.steps, ms, world)
+    e2e = aggregate_value(w.N, args.steps, ms_e2e, world)
     h2d, d2h = job.host_bytes_per_step()
     mix_ms = stage_ms["mix"] / max(stage_rounds, 1)
     achieved = job.mix_bytes_per_launch() / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
-    roofline = {"kernel": "mix_panel_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+    staged = w.weight_rule == "uniform" and 64 <= w.N <= 1024 and w.N * 128 > 113 * 1024
+    roofline = {"kernel": "mix_staged_kernel" if staged else "mix_panel_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind,
-                "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
+                "frac_of_8TBps_nominal": achieved / 8000.0,
+                "traffic": MIX_TRAFFIC_BYTES.get(args.config) if not (args.width or args.samples) else None,
                 "bytes_per_launch": job.mix_bytes_per_launch(), "ms_per_launch": mix_ms}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
