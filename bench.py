@@ -76,6 +76,7 @@ class Job:
                 labels[i].copy_(torch.from_numpy(l))
             self.feat, self.labels = feat, labels
             self.h.set_dataset(feat, labels, w.samples)
+            self.h.set_param_tracking(True)      # X is updated in place and never modified between rounds
             X0 = np.stack([wl.init_params(w, i) for i in range(w.N)])
             self.X = torch.from_numpy(self.m.pack(X0)).to(self.dev)
             self.G = None

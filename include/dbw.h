@@ -181,6 +181,16 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
               float* loss, void* stream);
 
 /*
+ * Parameter tracking for chained rounds (tensor-core path; a no-op otherwise).  Each round the
+ * BF16 GEMMs need a bf16 copy of the weights.  With tracking on, dbw_mix / dbw_round write that copy
+ * next to X' (same values as a later cast, so results do not change), and the next dbw_grad /
+ * dbw_round skips the cast when its X is the very X_out of the previous call.  The caller promises
+ * not to modify that buffer in between; if it does (or passes other parameters at the same
+ * address), it must turn tracking off and on again, which forgets the copy.  Off by default.
+ */
+int dbw_set_param_tracking(dbw_handle* h, int enable);
+
+/*
  * The same round for callers whose per-round inputs live in HOST memory (pinned memory makes
  * the copies asynchronous).  X / X_out / G_ext stay DEVICE (the parameters are the state of the
  * simulation); h_t[N], h_b[N], h_batch_idx[N][batch] are copied to the device on `stream`, the

@@ -295,6 +295,14 @@ int dbw_mix(dbw_handle* h, const float* X, const float* G, const uint8_t* kept, 
     return launch_mix(h, X, G, lr, lr_per_worker, X_out, (cudaStream_t)stream);
 }
 
+int dbw_set_param_tracking(dbw_handle* h, int enable) {
+    if (!h) return DBW_ERR_NULL;
+    h->track_params = enable != 0;
+    h->shadow_valid = false;
+    h->shadow_of = nullptr;
+    return DBW_OK;
+}
+
 int dbw_mix_in_place_ok(const dbw_handle* h) { return h && mix_panel_fits(h) ? 1 : 0; }
 
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols) {

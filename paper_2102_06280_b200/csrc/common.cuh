@@ -87,6 +87,13 @@ struct dbw_handle {
     int32_t* d_ylab = nullptr;              // [N][B] gathered labels
     float* d_G = nullptr;                   // [N][ld] gradient workspace of dbw_round (lazy)
     dbw::BF16State* bf16 = nullptr;
+    // bf16 shadow of the parameter matrix, [N][ld], same layout as X (tensor-core path only).  The
+    // mix writes it next to X' when parameter tracking is on; the next gradient call then skips the
+    // weight cast if it is handed that very X'.
+    uint16_t* d_shadow = nullptr;
+    bool track_params = false;
+    bool shadow_valid = false;
+    const float* shadow_of = nullptr;
 
     // stage timing (dbw_profile): events[round][stage boundary 0..3]
     bool profiling = false;
@@ -113,12 +120,19 @@ int launch_plan_from_kept(dbw_handle* h, const uint8_t* kept, const int32_t* b, 
 // mix.cu
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s);
+// device helper shared by the mix kernels: four floats -> four bf16 (round to nearest even)
+__device__ __forceinline__ uint2 pack_bf16x4_rn(float a, float b, float c, float d) {
+    uint32_t lo, hi;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(b), "f"(a));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(d), "f"(c));
+    return make_uint2(lo, hi);
+}
 bool mix_panel_fits(const dbw_handle* h);
 
 // mix_staged.cu
 bool mix_staged_usable(const dbw_handle* h);
 int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
-                      cudaStream_t s);
+                      uint16_t* shadow, cudaStream_t s);
 
 // dtur.cu
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);

@@ -299,8 +299,8 @@ cast_tile_kernel(int rows, int cols, const float* __restrict__ src, long long sr
                 const float4 f = __ldg(reinterpret_cast<const float4*>(p + e));
                 v[e] = f.x; v[e + 1] = f.y; v[e + 2] = f.z; v[e + 3] = f.w;
             }
-        if (c0 < cols) *reinterpret_cast<uint4*>(d) = pack8(v);
-        if (c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
+        if (dst && c0 < cols) *reinterpret_cast<uint4*>(d) = pack8(v);
+        if (dst && c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
     }
     if (!dstT) return;
 #pragma unroll
@@ -347,36 +347,83 @@ bias_grad_t_kernel(int out_dim, int B, const bf16* __restrict__ dzT, long long d
 constexpr int kMaxClasses = 32;
 
 // logits = A W^T + b (A bf16 [B][K], W fp32 master [C][K]), then dZ = (softmax - onehot)/B and the
-// per-sample loss.  One warp per sample.
-__global__ void __launch_bounds__(256)
+// per-sample loss.  A warp takes four samples at once: each lane owns 8 consecutive k of every
+// 256-wide chunk (one 128-bit load per sample, two per weight row), so a weight row fetched from
+// L1/L2 is used for four samples.
+template <int CP>
+__global__ void __launch_bounds__(128)
 head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld, long long w_off,
                     long long b_off, const int32_t* __restrict__ ylab, float* __restrict__ dzL, float* __restrict__ loss_s) {
     const int i = blockIdx.y;
-    const int s = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int s0 = (blockIdx.x * 4 + (threadIdx.x >> 5)) * 4;
     const int lane = threadIdx.x & 31;
-    if (s >= B) return;
-    const bf16* a = A + ((size_t)i * B + s) * K;
+    if (s0 >= B) return;
     const float* W = X + (size_t)i * ld + w_off;
-    float z_mine = 0.f;  // lane c ends up holding logit c
-    for (int c = 0; c < C; ++c) {
-        float acc = 0.f;
-        for (int k = lane; k < K; k += 32) acc = fmaf(__bfloat162float(a[k]), __ldg(W + (size_t)c * K + k), acc);
+    float acc[4][CP];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == c) z_mine = acc + X[(size_t)i * ld + b_off + c];
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[u][c] = 0.f;
+    auto load_a = [&](int kc, uint4 (&raw)[4]) {
+        const int k = kc + lane * 8;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (k < K && s0 + u < B) raw[u] = __ldg(reinterpret_cast<const uint4*>(A + ((size_t)i * B + s0 + u) * K + k));
+        }
+    };
+    uint4 cur[4], nxt[4];
+    load_a(0, cur);
+    for (int kc = 0; kc < K; kc += 256) {
+        load_a(kc + 256, nxt);  // next chunk in flight while this one is used (all zero past the end)
+        const int k = kc + lane * 8;
+        if (k < K) {
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                if (c < C) {
+                    const float4 w0 = __ldg(reinterpret_cast<const float4*>(W + (size_t)c * K + k));
+                    const float4 w1 = __ldg(reinterpret_cast<const float4*>(W + (size_t)c * K + k + 4));
+                    const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {  // bf16 -> fp32 is a 16-bit shift
+                            acc[u][c] = fmaf(__uint_as_float(w4[e] << 16), wv[2 * e], acc[u][c]);
+                            acc[u][c] = fmaf(__uint_as_float(w4[e] & 0xffff0000u), wv[2 * e + 1], acc[u][c]);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) cur[u] = nxt[u];
     }
-    const float zl = lane < C ? z_mine : -INFINITY;
-    float mx = zl;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    const float e = lane < C ? expf(zl - mx) : 0.f;
-    float sum = e;
+    for (int u = 0; u < 4; ++u) {
+        float z_mine = 0.f;  // lane c ends up holding logit c of sample s0 + u
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const int y = ylab[(size_t)i * B + s];
-    if (lane < C) dzL[((size_t)i * B + s) * C + lane] = (e / sum - (lane == y ? 1.f : 0.f)) / (float)B;
-    const float zy = __shfl_sync(0xffffffffu, zl, y & 31);
-    if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+        for (int c = 0; c < CP; ++c) {
+            float v = acc[u][c];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == c) z_mine = v;
+        }
+        const int s = s0 + u;
+        if (s >= B) continue;  // warp-uniform
+        const float zl = lane < C ? z_mine + X[(size_t)i * ld + b_off + lane] : -INFINITY;
+        float mx = zl;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float e = lane < C ? expf(zl - mx) : 0.f;
+        float sum = e;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const int y = ylab[(size_t)i * B + s];
+        if (lane < C) dzL[((size_t)i * B + s) * C + lane] = (e / sum - (lane == y ? 1.f : 0.f)) / (float)B;
+        const float zy = __shfl_sync(0xffffffffu, zl, y & 31);
+        if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+    }
 }
 
 __global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, float* __restrict__ loss) {
@@ -388,15 +435,17 @@ __global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, floa
     if (lane == 0) loss[i] = s / (float)B;
 }
 
-// Last layer backward; thread k of a block owns input feature k:
+// Last layer backward; a thread owns KPT consecutive input features k:
 //   dW[c][k] = sum_s dZ[s][c] A[s][k],  db[c] = sum_s dZ[s][c],
 //   dZprev[s][k] = [A[s][k] > 0] * sum_c dZ[s][c] W[c][k]   (bf16, plus its transpose [K][B]).
-template <int CP>
-__global__ void __launch_bounds__(128)
+// dZ of the worker sits in shared memory and is read as 128-bit broadcasts.
+template <int CP, int KPT>
+__global__ void __launch_bounds__(64)
 head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld,
                      long long w_off, long long b_off, const float* __restrict__ dzL, float* __restrict__ G,
                      bf16* __restrict__ dzP, bf16* __restrict__ dzPT) {
-    extern __shared__ float sdz[];  // [B][CP]
+    extern __shared__ float4 sdz4[];  // [B][CP] floats
+    float* sdz = reinterpret_cast<float*>(sdz4);
     const int i = blockIdx.y;
     for (int e = threadIdx.x; e < B * CP; e += blockDim.x) {
         const int s = e / CP, c = e % CP;
@@ -408,39 +457,82 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
         for (int s = 0; s < B; ++s) t += sdz[s * CP + threadIdx.x];
         G[(size_t)i * ld + b_off + threadIdx.x] = t;
     }
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= K) return;
-    float w[CP], dw[CP];
+    const int k = (blockIdx.x * 64 + threadIdx.x) * KPT;
+    if (k >= K) return;  // K % 8 == 0, so k + KPT <= K
+    float w[CP][KPT], dw[CP][KPT];
 #pragma unroll
-    for (int c = 0; c < CP; ++c) {
-        w[c] = c < C ? X[(size_t)i * ld + w_off + (size_t)c * K + k] : 0.f;
-        dw[c] = 0.f;
-    }
+    for (int c = 0; c < CP; ++c)
+#pragma unroll
+        for (int q = 0; q < KPT; ++q) {
+            w[c][q] = c < C ? X[(size_t)i * ld + w_off + (size_t)c * K + k + q] : 0.f;
+            dw[c][q] = 0.f;
+        }
     const bf16* a = A + (size_t)i * B * K + k;
+    auto load_a = [&](int s0, uint32_t (&raw)[8]) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            raw[u] = 0u;
+            if (s0 + u < B) {
+                if (KPT == 2)
+                    raw[u] = __ldg(reinterpret_cast<const uint32_t*>(a + (size_t)(s0 + u) * K));
+                else
+                    raw[u] = (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a + (size_t)(s0 + u) * K)) << 16;
+            }
+        }
+    };
+    uint32_t cur[8], nxt[8];
+    load_a(0, cur);
     for (int s0 = 0; s0 < B; s0 += 8) {  // B % 8 == 0
-        float dav[8];
+        load_a(s0 + 8, nxt);  // next eight samples in flight while these are used
+        float dav[KPT][8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int s = s0 + u;
-            const float av = __bfloat162float(a[(size_t)s * K]);
-            float da = 0.f;
-#pragma unroll
-            for (int c = 0; c < CP; ++c) {
-                const float dz = sdz[s * CP + c];
-                dw[c] = fmaf(dz, av, dw[c]);
-                da = fmaf(dz, w[c], da);
+            float av[KPT];
+            if (KPT == 2) {
+                av[0] = __uint_as_float(cur[u] << 16);
+                av[KPT - 1] = __uint_as_float(cur[u] & 0xffff0000u);
+            } else {
+                av[0] = __uint_as_float(cur[u]);
             }
-            dav[u] = av > 0.f ? da : 0.f;
-            if (dzP) dzP[((size_t)i * B + s) * K + k] = __float2bfloat16_rn(dav[u]);
+            float da[KPT];
+#pragma unroll
+            for (int q = 0; q < KPT; ++q) da[q] = 0.f;
+#pragma unroll
+            for (int c4 = 0; c4 < CP / 4; ++c4) {
+                const float4 d4 = sdz4[s * (CP / 4) + c4];
+                const float dz[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int q = 0; q < KPT; ++q) {
+                        dw[4 * c4 + e][q] = fmaf(dz[e], av[q], dw[4 * c4 + e][q]);
+                        da[q] = fmaf(dz[e], w[4 * c4 + e][q], da[q]);
+                    }
+            }
+#pragma unroll
+            for (int q = 0; q < KPT; ++q) dav[q][u] = av[q] > 0.f ? da[q] : 0.f;
+            if (dzP) {
+                if (KPT == 2)
+                    *reinterpret_cast<uint32_t*>(dzP + ((size_t)i * B + s) * K + k) = pack_bf16x2(dav[0][u], dav[KPT - 1][u]);
+                else
+                    dzP[((size_t)i * B + s) * K + k] = __float2bfloat16_rn(dav[0][u]);
+            }
         }
         if (dzPT)
-            *reinterpret_cast<uint4*>(dzPT + ((size_t)i * K + k) * B + s0) =
-                make_uint4(pack_bf16x2(dav[0], dav[1]), pack_bf16x2(dav[2], dav[3]), pack_bf16x2(dav[4], dav[5]),
-                           pack_bf16x2(dav[6], dav[7]));
+#pragma unroll
+            for (int q = 0; q < KPT; ++q)
+                *reinterpret_cast<uint4*>(dzPT + ((size_t)i * K + k + q) * B + s0) =
+                    make_uint4(pack_bf16x2(dav[q][0], dav[q][1]), pack_bf16x2(dav[q][2], dav[q][3]),
+                               pack_bf16x2(dav[q][4], dav[q][5]), pack_bf16x2(dav[q][6], dav[q][7]));
+#pragma unroll
+        for (int u = 0; u < 8; ++u) cur[u] = nxt[u];
     }
 #pragma unroll
     for (int c = 0; c < CP; ++c)
-        if (c < C) G[(size_t)i * ld + w_off + (size_t)c * K + k] = dw[c];
+        if (c < C)
+#pragma unroll
+            for (int q = 0; q < KPT; ++q) G[(size_t)i * ld + w_off + (size_t)c * K + k + q] = dw[c][q];
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -461,13 +553,14 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// K-major operand [workers][rows][K] bf16, dense: box = 64 (K) x 128 (rows) x 1, 128-byte swizzle,
+// K-major operand [workers][rows][K] bf16: box = 64 (K) x 128 (rows) x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
-bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers) {
+bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers, long long worker_pitch = 0) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    if (!worker_pitch) worker_pitch = (long long)K * rows;  // dense blocks unless the operand lives inside a wider row
     cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)workers};
-    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * 2 * (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)worker_pitch * 2};
     cuuint32_t box[3] = {BK, BM, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr,
@@ -480,7 +573,7 @@ bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int w
 struct BF16State {
     bf16* A[DBW_MAX_LAYERS] = {};    // A_l   [N][B][dims[l]],  l = 0..L-1
     bf16* AT[DBW_MAX_LAYERS] = {};   // A_l^T [N][dims[l]][B],  l = 0..L-2
-    bf16* Wh[DBW_MAX_LAYERS] = {};   // W_l   [N][out][in],     l = 0..L-2
+    bf16* Wh[DBW_MAX_LAYERS] = {};   // W_l   [out][in] inside the bf16 shadow rows (worker pitch ld), l = 0..L-2
     bf16* WhT[DBW_MAX_LAYERS] = {};  // W_l^T [N][in][out],     l = 1..L-2
     bf16* dZ[DBW_MAX_LAYERS] = {};   // dZ_l  [N][B][dims[l]],  l = 1..L-1
     bf16* dZT[DBW_MAX_LAYERS] = {};  // dZ_l^T
@@ -526,7 +619,6 @@ int grad_bf16_alloc(dbw_handle* h) {
         ok = ok && balloc(st, &st->A[l], NB * m.dims[l]);
         if (l <= L - 2) {
             ok = ok && balloc(st, &st->AT[l], NB * m.dims[l]);
-            ok = ok && balloc(st, &st->Wh[l], (size_t)N * m.dims[l] * m.dims[l + 1]);
             if (l >= 1) ok = ok && balloc(st, &st->WhT[l], (size_t)N * m.dims[l] * m.dims[l + 1]);
         }
         if (l >= 1) {
@@ -534,11 +626,15 @@ int grad_bf16_alloc(dbw_handle* h) {
             ok = ok && balloc(st, &st->dZT[l], NB * m.dims[l]);
         }
     }
+    bf16* shadow = nullptr;
+    ok = ok && balloc(st, &shadow, (size_t)N * h->ld);
+    h->d_shadow = reinterpret_cast<uint16_t*>(shadow);
+    for (int l = 0; l <= L - 2 && ok; ++l) st->Wh[l] = shadow + m.w_off[l];
     ok = ok && balloc(st, &st->dzL, NB * m.dims[L]) && balloc(st, &st->loss_s, NB) && balloc(st, &st->ylab, NB);
     if (!ok) return DBW_ERR_CUDA;
     for (int l = 0; l <= L - 2; ++l) {
         ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
-        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N);
+        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld);
         ok = ok && make_operand_map(&st->dwA[l], st->dZT[l + 1], B, m.dims[l + 1], N);
         ok = ok && make_operand_map(&st->dwB[l], st->AT[l], B, m.dims[l], N);
         if (l >= 1) {
@@ -548,13 +644,14 @@ int grad_bf16_alloc(dbw_handle* h) {
     }
     if (!ok) return DBW_ERR_CUDA;
     DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
-    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
 }
 
 void grad_bf16_free(dbw_handle* h) {
     if (!h->bf16) return;
+    h->d_shadow = nullptr;
     for (void* p : h->bf16->owned) cudaFree(p);
     delete h->bf16;
     h->bf16 = nullptr;
@@ -565,12 +662,16 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     BF16State* st = h->bf16;
     const int L = m.n_layers, B = m.batch, N = h->N, C = m.dims[L];
     int rc;
-    // bf16 copies of the weights of the tensor-core layers (and their transposes for dA)
+    // bf16 copies of the weights of the tensor-core layers (inside the shadow rows) and their
+    // transposes for dA.  When the previous mix already wrote the shadow of this very X, only the
+    // transposes are left to do.
+    const bool have_shadow = h->track_params && h->shadow_valid && h->shadow_of == X;
     for (int l = 0; l <= L - 2; ++l) {
         const int in = m.dims[l], out = m.dims[l + 1];
+        if (have_shadow && l == 0) continue;
         cast_tile_kernel<<<dim3((in + 63) / 64, (out + 63) / 64, N), 256, 0, s>>>(
-            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], (long long)in * out, l >= 1 ? st->WhT[l] : nullptr,
-            (long long)in * out, h->d_status);
+            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, have_shadow ? nullptr : st->Wh[l], h->ld,
+            l >= 1 ? st->WhT[l] : nullptr, (long long)in * out, h->d_status);
         DBW_LAUNCHED();
     }
     // mini-batch gather: A_0 (and A_0^T when a tensor-core layer consumes it)
@@ -592,8 +693,12 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     }
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
-    head_forward_kernel<<<dim3((B + 7) / 8, N), 256, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1],
-                                                             st->ylab, st->dzL, st->loss_s);
+    if (C <= 16)
+        head_forward_kernel<16><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+                                                                       m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
+    else
+        head_forward_kernel<32><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+                                                                       m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     DBW_LAUNCHED();
     if (loss) {
         loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
@@ -602,10 +707,10 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
     bf16* dzPT = L >= 2 ? st->dZT[L - 1] : nullptr;
     if (C <= 16)
-        head_backward_kernel<16><<<dim3((K + 127) / 128, N), 128, (size_t)B * 16 * 4, s>>>(
+        head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N), 64, (size_t)B * 16 * 4, s>>>(
             B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
     else
-        head_backward_kernel<32><<<dim3((K + 127) / 128, N), 128, (size_t)B * 32 * 4, s>>>(
+        head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N), 64, (size_t)B * 32 * 4, s>>>(
             B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
     DBW_LAUNCHED();
     // backward through the tensor-core layers

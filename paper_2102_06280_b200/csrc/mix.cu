@@ -27,8 +27,8 @@ __device__ __forceinline__ float4 fma4(float w, float4 v, float4 a) {
 template <int GS>
 __global__ void __launch_bounds__(kMixThreads)
 mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ G, float lr,
-                 const float* __restrict__ lr_pw, float* Xout, MixPlan plan, int mix_then_correct,
-                 int n_panels) {
+                 const float* __restrict__ lr_pw, float* Xout, uint16_t* __restrict__ shadow, MixPlan plan,
+                 int mix_then_correct, int n_panels) {
     extern __shared__ float4 sm[];  // [N][GS]
     const int tid = threadIdx.x;
     const int q = tid % GS;
@@ -78,6 +78,7 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
                     acc = fma4(-(lr_pw ? lr_pw[i] : lr), g, acc);
                 }
                 *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
+                if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
             }
         }
         __syncthreads();
@@ -88,8 +89,8 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
 // neighbour rows re-read through L2.  Out of place only.
 __global__ void __launch_bounds__(256)
 mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float* __restrict__ G, float lr,
-                  const float* __restrict__ lr_pw, float* __restrict__ Xout, MixPlan plan,
-                  int mix_then_correct) {
+                  const float* __restrict__ lr_pw, float* __restrict__ Xout, uint16_t* __restrict__ shadow,
+                  MixPlan plan, int mix_then_correct) {
     const long long ld4 = ld / 4;
     const long long total = (long long)N * ld4;
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
@@ -111,6 +112,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
             acc = fma4(plan.w[(size_t)i * plan.stride + k], stepped(plan.idx[(size_t)i * plan.stride + k]), acc);
         if (mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
         *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
+        if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
     }
 }
 
@@ -127,7 +129,7 @@ int auto_group_size(const dbw_handle* h) {
 
 template <int GS>
 int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
-                 cudaStream_t s) {
+                 uint16_t* shadow, cudaStream_t s) {
     const size_t smem = (size_t)h->N * GS * 16;
     static bool configured[64] = {};
     if (!configured[h->device & 63]) {
@@ -140,7 +142,7 @@ int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const 
     if (per_sm < 1) return DBW_ERR_BAD_SHAPE;
     const int n_panels = (int)((h->ld + 4 * GS - 1) / (4 * GS));
     const int grid = n_panels < per_sm * h->sm_count ? n_panels : per_sm * h->sm_count;
-    mix_panel_kernel<GS><<<grid, kMixThreads, smem, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, h->plan,
+    mix_panel_kernel<GS><<<grid, kMixThreads, smem, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, shadow, h->plan,
                                                         (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0,
                                                         n_panels);
     DBW_LAUNCHED();
@@ -161,12 +163,17 @@ bool mix_panel_fits(const dbw_handle* h) { return use_staged(h) || auto_group_si
 
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s) {
-    if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, s);
+    // With parameter tracking the bf16 shadow of X' is written alongside; any other mix call leaves
+    // the shadow stale for the buffer it describes.
+    uint16_t* shadow = (h->track_params && h->d_shadow) ? h->d_shadow : nullptr;
+    h->shadow_valid = shadow != nullptr;
+    h->shadow_of = X_out;
+    if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, shadow, s);
     switch (auto_group_size(h)) {
-        case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, s);
-        case 16: return launch_panel<16>(h, X, G, lr, lr_pw, X_out, s);
-        case 8: return launch_panel<8>(h, X, G, lr, lr_pw, X_out, s);
-        case 4: return launch_panel<4>(h, X, G, lr, lr_pw, X_out, s);
+        case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, shadow, s);
+        case 16: return launch_panel<16>(h, X, G, lr, lr_pw, X_out, shadow, s);
+        case 8: return launch_panel<8>(h, X, G, lr, lr_pw, X_out, shadow, s);
+        case 4: return launch_panel<4>(h, X, G, lr, lr_pw, X_out, shadow, s);
         default: break;
     }
     if (X_out == X) return DBW_ERR_BAD_SHAPE;
@@ -174,7 +181,7 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
     long long blocks = (total + 255) / 256;
     const long long cap = (long long)h->sm_count * 8;
     if (blocks > cap) blocks = cap;
-    mix_direct_kernel<<<(int)blocks, 256, 0, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, h->plan,
+    mix_direct_kernel<<<(int)blocks, 256, 0, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, shadow, h->plan,
                                                  (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0);
     DBW_LAUNCHED();
     return DBW_OK;

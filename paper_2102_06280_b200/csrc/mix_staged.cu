@@ -63,6 +63,7 @@ struct StagedArgs {
     float lr;
     const float* lr_pw;
     float* Xout;
+    uint16_t* shadow;
     MixPlan plan;
 };
 
@@ -184,6 +185,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
                     acc.z = fmaf(nlr, gi.z, acc.z); acc.w = fmaf(nlr, gi.w, acc.w);
                 }
                 *reinterpret_cast<float4*>(a.Xout + (size_t)i * a.ld + c) = acc;
+                if (a.shadow) *reinterpret_cast<uint2*>(a.shadow + (size_t)i * a.ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
             }
         }
     };
@@ -237,14 +239,14 @@ bool mix_staged_usable(const dbw_handle* h) {
 }
 
 int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
-                      cudaStream_t s) {
+                      uint16_t* shadow, cudaStream_t s) {
     StagedArgs a{};
     a.N = h->N;
     a.ld = h->ld;
     a.n_panels = (int)((h->ld + 31) / 32);
     a.mix_then_correct = (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0;
     a.plan_row = (h->maxdeg + 7) / 8 * 8;
-    a.X = X; a.G = G; a.lr = lr; a.lr_pw = lr_pw; a.Xout = X_out; a.plan = h->plan;
+    a.X = X; a.G = G; a.lr = lr; a.lr_pw = lr_pw; a.Xout = X_out; a.shadow = shadow; a.plan = h->plan;
     const size_t smem = staged_smem(h, a.plan_row);
     static bool configured[64] = {};
     if (!configured[h->device & 63]) {

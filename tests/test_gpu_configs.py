@@ -154,6 +154,7 @@ def _free_run_bf16(w, rounds):
     own neighbours in parameter space just as well.  Masks, times, b and theta stay bit-exact."""
     import paper_2102_06280_b200 as p
     sim = Sim(w, p.GEMM_BF16)
+    sim.h.set_param_tracking(True)      # X_gpu is updated in place and never touched in between
     m = sim.m
     times = wl.arrival_times(w, rounds)
     X_gpu = dev(m.pack(sim.X0))
@@ -178,6 +179,38 @@ def _free_run_bf16(w, rounds):
     assert mx <= 5e-2, mx              # element-wise: bf16 rounding flips ReLU masks near zero
     assert sim.h.status() == 0
     sim.h.close()
+
+
+def test_param_tracking_is_bitwise_neutral():
+    """With tracking on, the mix writes the bf16 weight copy that the next round's GEMMs read; the
+    values are those of a cast after the fact, so four chained rounds give the same bits either way."""
+    import paper_2102_06280_b200 as p
+    w = wl.make_workload(2, N=16, er_p=0.35, samples=300)
+    times = wl.arrival_times(w, 4)
+    outs = []
+    for track in (False, True):
+        sim = Sim(w, p.GEMM_BF16)
+        sim.h.set_param_tracking(track)
+        X = dev(sim.m.pack(sim.X0))
+        for k in range(4):
+            sim.backups(k, times[k])
+            sim.gpu_round(X, times[k], wl.batch_indices(w, k), X)
+        outs.append(X.clone())
+        # a caller that changes the parameters behind the library's back must reset tracking
+        if track:
+            X.mul_(0.5)
+            sim.h.set_param_tracking(False)
+            sim.h.set_param_tracking(True)
+            sim.gpu_round(X, times[0], wl.batch_indices(w, 0), X)
+            ref = Sim(w, p.GEMM_BF16)
+            ref.b_d.copy_(sim.b_d)
+            Y = (outs[1] * 0.5).contiguous()
+            ref.gpu_round(Y, times[0], wl.batch_indices(w, 0), Y)
+            assert torch.equal(X, Y)
+            ref.h.close()
+        assert sim.h.status() == 0
+        sim.h.close()
+    assert torch.equal(outs[0], outs[1])
 
 
 def test_config2_bf16_free_running_20_rounds():
