@@ -104,12 +104,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ bool bf16_bits_positive(uint32_t bits16) { return (bits16 & 0x8000u) == 0 && (bits16 & 0x7fffu) != 0; }
 
 // ----------------------------------------------------------------------------- tensor-core GEMM
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3, UMMA_K = 16;
-constexpr int TILE_BYTES = BM * BK * 2;  // 16 KiB per operand tile
+constexpr int BM = 128, BK = 64, UMMA_K = 16;  // tile: 128 rows x BN columns (128 or 256) x 64 deep
+constexpr int TILE_BYTES = BM * BK * 2;  // 16 KiB per 128-row operand tile
 constexpr int GEMM_THREADS = 192;
-constexpr size_t GEMM_SMEM = (size_t)STAGES * 2 * TILE_BYTES + 1024 /*align slack*/ + 128 /*barriers*/;
-// kind::f16, D = f32, A = B = bf16, both K-major, N = 128, M = 128
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr size_t gemm_smem(int stages, int bn) { return (size_t)stages * (TILE_BYTES + bn * BK * 2) + 1024 /*align slack*/ + 128 /*barriers*/; }
+// kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = bn
+__host__ __device__ constexpr uint32_t idesc_for(int bn) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24); }
 
 enum { EPI_FWD = 0, EPI_DA = 1, EPI_DW = 2 };
 
@@ -123,13 +123,16 @@ struct TcArgs {
     uint32_t* status;
 };
 
+template <int STAGES, int BN>
 __global__ void __launch_bounds__(GEMM_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* tilesA = smem;
+    constexpr int TILE_B_BYTES = BN * BK * 2;
+    constexpr uint32_t IDESC = idesc_for(BN);
     uint8_t* tilesB = smem + STAGES * TILE_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + 2 * STAGES * TILE_BYTES);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * (TILE_BYTES + TILE_B_BYTES));
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
@@ -160,9 +163,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % STAGES;
                 if (kb >= STAGES) mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1, g.status);
-                mbar_expect_tx(&full[s], 2 * TILE_BYTES);
+                mbar_expect_tx(&full[s], TILE_BYTES + TILE_B_BYTES);
                 tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
-                tma_load_3d(tilesB + s * TILE_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+                tma_load_3d(tilesB + s * TILE_B_BYTES, &tmB, kb * BK, n0, z, &full[s]);
             }
         }
     } else if (warp == 1) {
@@ -172,7 +175,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 mbar_wait(&full[s], (kb / STAGES) & 1, g.status);
                 tc_fence_after();
                 const uint64_t da = kmajor_sw128_desc(smem_u32(tilesA + s * TILE_BYTES));
-                const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_BYTES));
+                const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_B_BYTES));
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes further along K inside the swizzle atom
                     tc_mma_bf16(tmem_base, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
@@ -555,13 +558,14 @@ EncodeTiledFn encode_fn() {
 
 // K-major operand [workers][rows][K] bf16: box = 64 (K) x 128 (rows) x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
-bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers, long long worker_pitch = 0) {
+bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers, long long worker_pitch = 0,
+                      int box_rows = BM) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     if (!worker_pitch) worker_pitch = (long long)K * rows;  // dense blocks unless the operand lives inside a wider row
     cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)workers};
     cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)worker_pitch * 2};
-    cuuint32_t box[3] = {BK, BM, 1};
+    cuuint32_t box[3] = {BK, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -593,9 +597,23 @@ bool balloc(BF16State* st, T** p, size_t n) {
     return true;
 }
 
+// Tile width for an output with N columns: 256 halves the operand re-reads out of L2 per output byte.
+int tile_bn(int N) { return N >= 256 ? 256 : 128; }
+
 int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
-    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, workers);
-    gemm_tc_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(a, b, g);
+    const int bn = tile_bn(g.N);
+    dim3 grid((g.N + bn - 1) / bn, (g.M + BM - 1) / BM, workers);
+    // short reductions (K <= 256: the dW GEMMs) take a two-stage ring so that more CTAs share an SM
+    // and one tile's epilogue overlaps the loads and MMAs of the others
+    const bool short_k = g.K <= 4 * BK;
+    if (bn == 128 && short_k)
+        gemm_tc_kernel<2, 128><<<grid, GEMM_THREADS, gemm_smem(2, 128), s>>>(a, b, g);
+    else if (bn == 128)
+        gemm_tc_kernel<3, 128><<<grid, GEMM_THREADS, gemm_smem(3, 128), s>>>(a, b, g);
+    else if (short_k)
+        gemm_tc_kernel<2, 256><<<grid, GEMM_THREADS, gemm_smem(2, 256), s>>>(a, b, g);
+    else
+        gemm_tc_kernel<2, 256><<<grid, GEMM_THREADS, gemm_smem(2, 256), s>>>(a, b, g);
     DBW_LAUNCHED();
     return DBW_OK;
 }
@@ -634,16 +652,18 @@ int grad_bf16_alloc(dbw_handle* h) {
     if (!ok) return DBW_ERR_CUDA;
     for (int l = 0; l <= L - 2; ++l) {
         ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
-        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld);
+        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1]));
         ok = ok && make_operand_map(&st->dwA[l], st->dZT[l + 1], B, m.dims[l + 1], N);
-        ok = ok && make_operand_map(&st->dwB[l], st->AT[l], B, m.dims[l], N);
+        ok = ok && make_operand_map(&st->dwB[l], st->AT[l], B, m.dims[l], N, 0, tile_bn(m.dims[l]));
         if (l >= 1) {
             ok = ok && make_operand_map(&st->daA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
-            ok = ok && make_operand_map(&st->daB[l], st->WhT[l], m.dims[l + 1], m.dims[l], N);
+            ok = ok && make_operand_map(&st->daB[l], st->WhT[l], m.dims[l + 1], m.dims[l], N, 0, tile_bn(m.dims[l]));
         }
     }
     if (!ok) return DBW_ERR_CUDA;
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2, 128)));
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 128)));
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2, 256)));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
