@@ -106,8 +106,11 @@ __device__ __forceinline__ bool bf16_bits_positive(uint32_t bits16) { return (bi
 // ----------------------------------------------------------------------------- tensor-core GEMM
 constexpr int BM = 128, BK = 64, UMMA_K = 16;  // tile: 128 rows x BN columns (128 or 256) x 64 deep
 constexpr int TILE_BYTES = BM * BK * 2;  // 16 KiB per 128-row operand tile
-constexpr int GEMM_THREADS = 192;
-constexpr size_t gemm_smem(int stages, int bn) { return (size_t)stages * (TILE_BYTES + bn * BK * 2) + 1024 /*align slack*/ + 128 /*barriers*/; }
+constexpr int GEMM_THREADS = 320;  // TMA warp, MMA warp, eight epilogue warps (two per accumulator lane quarter)
+constexpr int EPI_WARPS = 8;
+constexpr size_t gemm_smem(int stages, int bn) {
+    return (size_t)stages * (TILE_BYTES + bn * BK * 2) + 8 * 32 * 36 * 4 /*epilogue staging*/ + 1024 /*align slack*/ + 256 /*barriers*/;
+}
 // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = bn
 __host__ __device__ constexpr uint32_t idesc_for(int bn) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24); }
 
@@ -123,22 +126,34 @@ struct TcArgs {
     uint32_t* status;
 };
 
-template <int STAGES, int BN>
-__global__ void __launch_bounds__(GEMM_THREADS)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs g) {
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+constexpr int STAGING_FLOATS = EPI_WARPS * 32 * 36;  // per epilogue warp a 32 x 32 fp32 block, rows 36 words apart
+
+// Persistent, warp-specialised GEMM: one CTA per SM walks the tiles (n fastest, then m, then worker).
+// Warp 0 streams operand tiles by TMA through a STAGES-deep ring, warp 1 issues the MMAs into one of
+// ACC accumulator buffers in tensor memory, warps 2-9 drain a finished buffer through the epilogue
+// while the next tile's loads and MMAs are already running.
+template <int STAGES, int BN, int ACC>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs g, int tiles_m,
+               int tiles_n, int n_tiles) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* tilesA = smem;
     constexpr int TILE_B_BYTES = BN * BK * 2;
     constexpr uint32_t IDESC = idesc_for(BN);
+    uint8_t* tilesA = smem;
     uint8_t* tilesB = smem + STAGES * TILE_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * (TILE_BYTES + TILE_B_BYTES));
+    float* staging = reinterpret_cast<float*>(smem + STAGES * (TILE_BYTES + TILE_B_BYTES));
+    uint64_t* full = reinterpret_cast<uint64_t*>(staging + STAGING_FLOATS);
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    uint64_t* acc_empty = acc_full + ACC;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + ACC);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
     const int num_kb = (g.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
@@ -146,11 +161,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(acc_full, 1);
+        for (int b = 0; b < ACC; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], EPI_WARPS);  // one arrival per epilogue warp
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(ACC * BN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -160,105 +178,129 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                if (kb >= STAGES) mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1, g.status);
-                mbar_expect_tx(&full[s], TILE_BYTES + TILE_B_BYTES);
-                tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
-                tma_load_3d(tilesB + s * TILE_B_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+            int it = 0;  // k-blocks issued so far, over all tiles of this CTA
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+                const int n0 = (tile % tiles_n) * BN, m0 = ((tile / tiles_n) % tiles_m) * BM, z = tile / (tiles_n * tiles_m);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (it >= STAGES) mbar_wait(&empty[s], ((it / STAGES) - 1) & 1, g.status);
+                    mbar_expect_tx(&full[s], TILE_BYTES + TILE_B_BYTES);
+                    tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
+                    tma_load_3d(tilesB + s * TILE_B_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                mbar_wait(&full[s], (kb / STAGES) & 1, g.status);
-                tc_fence_after();
-                const uint64_t da = kmajor_sw128_desc(smem_u32(tilesA + s * TILE_BYTES));
-                const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_B_BYTES));
+            int it = 0, lt = 0;
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++lt) {
+                const int buf = lt % ACC;
+                if (lt >= ACC) {  // the epilogue must have drained this buffer's previous tile
+                    mbar_wait(&acc_empty[buf], ((lt / ACC) - 1) & 1, g.status);
+                    tc_fence_after();
+                }
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    mbar_wait(&full[s], (it / STAGES) & 1, g.status);
+                    tc_fence_after();
+                    const uint64_t da = kmajor_sw128_desc(smem_u32(tilesA + s * TILE_BYTES));
+                    const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_B_BYTES));
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes further along K inside the swizzle atom
-                    tc_mma_bf16(tmem_base, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
-                                (kb > 0 || k > 0) ? 1u : 0u);
-                tc_commit(&empty[s]);  // frees the stage once these MMAs have read it
+                    for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes further along K inside the swizzle atom
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
+                                    (kb > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(&empty[s]);  // frees the stage once these MMAs have read it
+                }
+                tc_commit(&acc_full[buf]);
             }
-            tc_commit(acc_full);
         }
     } else {
-        // ---- epilogue: warp w owns accumulator lanes 32*(w%4) .. +31, i.e. those output rows ----
-        mbar_wait(acc_full, 0, g.status);
-        tc_fence_after();
+        // ---- epilogue: warp w owns accumulator lanes 32*(w%4) .. +31, i.e. those output rows, and
+        // one half of the tile's columns (two warps share a lane quarter) ----
         const int q = warp & 3;
-        const int m = m0 + q * 32 + lane;
-        const bool m_ok = m < g.M;
-        for (int c = 0; c < BN / 32; ++c) {
-            const int nb = n0 + c * 32;
-            if (nb >= g.N) break;  // warp-uniform
-            uint32_t r[32];
-            tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
-            if (g.epi == EPI_DW) {
-                // Each lane holds one row of a 32 x 32 fp32 block.  It goes through shared memory (the
-                // drained pipeline stages; rows 36 words apart keep both 128-bit phases conflict-free)
-                // so that a warp stores four full 128-byte lines per instruction.
-                float* stg = reinterpret_cast<float*>(smem) + q * (32 * 36);
+        const int half = (warp - 2) >> 2;
+        float* stg = staging + (warp - 2) * (32 * 36);
+        int lt = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++lt) {
+            const int n0 = (tile % tiles_n) * BN, m0 = ((tile / tiles_n) % tiles_m) * BM, z = tile / (tiles_n * tiles_m);
+            const int buf = lt % ACC;
+            mbar_wait(&acc_full[buf], (lt / ACC) & 1, g.status);
+            tc_fence_after();
+            const int m = m0 + q * 32 + lane;
+            const bool m_ok = m < g.M;
+            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+                const int nb = n0 + c * 32;
+                if (nb >= g.N) break;  // warp-uniform
+                uint32_t r[32];
+                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
+                if (g.epi == EPI_DW) {
+                    // Each lane holds one row of a 32 x 32 fp32 block.  It goes through shared memory
+                    // (rows 36 words apart keep both 128-bit phases conflict-free) so that a warp
+                    // stores four full 128-byte lines per instruction.
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<uint4*>(stg + lane * 36 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-                __syncwarp();
-                const int f4 = lane & 7;
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<uint4*>(stg + lane * 36 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                    __syncwarp();
+                    const int f4 = lane & 7;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int row = 4 * i + (lane >> 3);
-                    const int mm = m0 + q * 32 + row;
-                    const float4 val = *reinterpret_cast<const float4*>(stg + row * 36 + 4 * f4);
-                    if (mm < g.M && nb + 4 * f4 < g.N)
-                        *reinterpret_cast<float4*>(g.outf + (size_t)z * g.outf_z + (size_t)mm * g.outf_pitch + nb + 4 * f4) = val;
-                }
-                __syncwarp();
-                continue;
-            }
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (g.epi == EPI_FWD) {
-                const float* bias = g.bias + (size_t)z * g.bias_z + nb;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + ((nb + j < g.N) ? __ldg(bias + j) : 0.f), 0.f);
-            } else if (m_ok) {  // EPI_DA: ReLU'(z) = [a > 0]
-                const bf16* mk = g.mask + (size_t)z * g.mask_z + (size_t)m * g.mask_pitch + nb;
-#pragma unroll
-                for (int j = 0; j < 32; j += 8)
-                    if (nb + j < g.N) {
-                        const uint4 u = __ldg(reinterpret_cast<const uint4*>(mk + j));
-                        const uint32_t wds[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            if (!bf16_bits_positive((wds[e >> 1] >> (16 * (e & 1))) & 0xffffu)) v[j + e] = 0.f;
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = 4 * i + (lane >> 3);
+                        const int mm = m0 + q * 32 + row;
+                        const float4 val = *reinterpret_cast<const float4*>(stg + row * 36 + 4 * f4);
+                        if (mm < g.M && nb + 4 * f4 < g.N)
+                            *reinterpret_cast<float4*>(g.outf + (size_t)z * g.outf_z + (size_t)mm * g.outf_pitch + nb + 4 * f4) = val;
                     }
-            }
-            uint32_t o[16];
+                    __syncwarp();
+                    continue;
+                }
+                float v[32];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
-            if (m_ok) {
-                bf16* dst = g.out + (size_t)z * g.out_z + (size_t)m * g.out_pitch + nb;
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                if (g.epi == EPI_FWD) {
+                    const float* bias = g.bias + (size_t)z * g.bias_z + nb;
 #pragma unroll
-                for (int j = 0; j < 32; j += 8)
-                    if (nb + j < g.N)
-                        *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[j / 2], o[j / 2 + 1], o[j / 2 + 2], o[j / 2 + 3]);
-                if (g.outT) {
-                    unsigned short* dt = reinterpret_cast<unsigned short*>(g.outT + (size_t)z * g.outT_z + (size_t)nb * g.outT_pitch + m);
+                    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + ((nb + j < g.N) ? __ldg(bias + j) : 0.f), 0.f);
+                } else if (m_ok) {  // EPI_DA: ReLU'(z) = [a > 0]
+                    const bf16* mk = g.mask + (size_t)z * g.mask_z + (size_t)m * g.mask_pitch + nb;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (nb + j < g.N) dt[(size_t)j * g.outT_pitch] = (unsigned short)((o[j >> 1] >> (16 * (j & 1))) & 0xffffu);
+                    for (int j = 0; j < 32; j += 8)
+                        if (nb + j < g.N) {
+                            const uint4 u = __ldg(reinterpret_cast<const uint4*>(mk + j));
+                            const uint32_t wds[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                if (!bf16_bits_positive((wds[e >> 1] >> (16 * (e & 1))) & 0xffffu)) v[j + e] = 0.f;
+                        }
+                }
+                uint32_t o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+                if (m_ok) {
+                    bf16* dst = g.out + (size_t)z * g.out_z + (size_t)m * g.out_pitch + nb;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        if (nb + j < g.N)
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[j / 2], o[j / 2 + 1], o[j / 2 + 2], o[j / 2 + 3]);
+                    if (g.outT) {
+                        unsigned short* dt = reinterpret_cast<unsigned short*>(g.outT + (size_t)z * g.outT_z + (size_t)nb * g.outT_pitch + m);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < g.N) dt[(size_t)j * g.outT_pitch] = (unsigned short)((o[j >> 1] >> (16 * (j & 1))) & 0xffffu);
+                    }
                 }
             }
+            // this warp's reads of the buffer are complete (tcgen05.wait::ld): hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(ACC * BN) : "memory");
     }
 }
 
@@ -600,20 +642,17 @@ bool balloc(BF16State* st, T** p, size_t n) {
 // Tile width for an output with N columns: 256 halves the operand re-reads out of L2 per output byte.
 int tile_bn(int N) { return N >= 256 ? 256 : 128; }
 
+int g_tc_sm_count = 0;
+
 int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
     const int bn = tile_bn(g.N);
-    dim3 grid((g.N + bn - 1) / bn, (g.M + BM - 1) / BM, workers);
-    // short reductions (K <= 256: the dW GEMMs) take a two-stage ring so that more CTAs share an SM
-    // and one tile's epilogue overlaps the loads and MMAs of the others
-    const bool short_k = g.K <= 4 * BK;
-    if (bn == 128 && short_k)
-        gemm_tc_kernel<2, 128><<<grid, GEMM_THREADS, gemm_smem(2, 128), s>>>(a, b, g);
-    else if (bn == 128)
-        gemm_tc_kernel<3, 128><<<grid, GEMM_THREADS, gemm_smem(3, 128), s>>>(a, b, g);
-    else if (short_k)
-        gemm_tc_kernel<2, 256><<<grid, GEMM_THREADS, gemm_smem(2, 256), s>>>(a, b, g);
+    const int tiles_n = (g.N + bn - 1) / bn, tiles_m = (g.M + BM - 1) / BM;
+    const int n_tiles = tiles_n * tiles_m * workers;
+    const int grid = n_tiles < g_tc_sm_count ? n_tiles : g_tc_sm_count;
+    if (bn == 128)
+        gemm_tc_kernel<4, 128, 2><<<grid, GEMM_THREADS, gemm_smem(4, 128), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
     else
-        gemm_tc_kernel<2, 256><<<grid, GEMM_THREADS, gemm_smem(2, 256), s>>>(a, b, g);
+        gemm_tc_kernel<3, 256, 2><<<grid, GEMM_THREADS, gemm_smem(3, 256), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
     DBW_LAUNCHED();
     return DBW_OK;
 }
@@ -661,9 +700,9 @@ int grad_bf16_alloc(dbw_handle* h) {
         }
     }
     if (!ok) return DBW_ERR_CUDA;
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2, 128)));
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 128)));
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2, 256)));
+    g_tc_sm_count = h->sm_count;
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<4, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(4, 128)));
+    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 256)));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
