@@ -46,46 +46,60 @@ struct GemmArgs {
     int relu;
 };
 
-constexpr int TM = 64, TN = 64, TK = 16;
+constexpr int TK = 16;
 
+// 256 threads, each an R x R micro-tile: tiles of 64 x 64 (R = 4) for large outputs, 32 x 32 (R = 2)
+// when the larger tile would leave most SMs idle.
+template <int R>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
-    __shared__ __align__(16) float As[TK][TM + 4];
-    __shared__ __align__(16) float Bs[TK][TN + 4];
+    constexpr int T = 16 * R;        // tile edge
+    constexpr int PER = T * TK / 256;  // elements of each operand tile a thread stages
+    __shared__ __align__(16) float As[TK][T + 4];
+    __shared__ __align__(16) float Bs[TK][T + 4];
     const int z = blockIdx.z;
-    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+    const int m0 = blockIdx.y * T, n0 = blockIdx.x * T;
     const float* A = g.A + (size_t)z * g.sAz;
     const float* B = g.B + (size_t)z * g.sBz;
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const bool a_k_fast = g.sAk == 1;
     const bool b_k_fast = g.sBk == 1;
-    float acc[4][4] = {};
+    float acc[R][R] = {};
+    float pa[PER], pb[PER];  // next k-step's operand elements, in flight while this one is multiplied
+    auto fetch = [&](int k0) {
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+            const int e = tid + r * 256;
+            const int ka = a_k_fast ? (e & 15) : (e / T);
+            const int ma = a_k_fast ? (e >> 4) : (e % T);
+            pa[r] = (m0 + ma < g.M && k0 + ka < g.K) ? __ldg(A + (size_t)(m0 + ma) * g.sAm + (size_t)(k0 + ka) * g.sAk) : 0.f;
+            const int kb = b_k_fast ? (e & 15) : (e / T);
+            const int nb = b_k_fast ? (e >> 4) : (e % T);
+            pb[r] = (n0 + nb < g.N && k0 + kb < g.K) ? __ldg(B + (size_t)(n0 + nb) * g.sBn + (size_t)(k0 + kb) * g.sBk) : 0.f;
+        }
+    };
+    fetch(0);
     for (int k0 = 0; k0 < g.K; k0 += TK) {
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
+        for (int r = 0; r < PER; ++r) {
             const int e = tid + r * 256;
-            const int ka = a_k_fast ? (e & 15) : (e >> 6);
-            const int ma = a_k_fast ? (e >> 4) : (e & 63);
-            float v = 0.f;
-            if (m0 + ma < g.M && k0 + ka < g.K) v = __ldg(A + (size_t)(m0 + ma) * g.sAm + (size_t)(k0 + ka) * g.sAk);
-            As[ka][ma] = v;
-            const int kb = b_k_fast ? (e & 15) : (e >> 6);
-            const int nb = b_k_fast ? (e >> 4) : (e & 63);
-            v = 0.f;
-            if (n0 + nb < g.N && k0 + kb < g.K) v = __ldg(B + (size_t)(n0 + nb) * g.sBn + (size_t)(k0 + kb) * g.sBk);
-            Bs[kb][nb] = v;
+            As[a_k_fast ? (e & 15) : (e / T)][a_k_fast ? (e >> 4) : (e % T)] = pa[r];
+            Bs[b_k_fast ? (e & 15) : (e / T)][b_k_fast ? (e >> 4) : (e % T)] = pb[r];
         }
         __syncthreads();
+        fetch(k0 + TK);  // all zero past the end
 #pragma unroll
         for (int kk = 0; kk < TK; ++kk) {
-            const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-            const float bv[4] = {b.x, b.y, b.z, b.w};
+            float av[R], bv[R];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < R; ++i) {
+                av[i] = As[kk][ty * R + i];
+                bv[i] = Bs[kk][tx * R + i];
+            }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+            for (int i = 0; i < R; ++i)
+#pragma unroll
+                for (int j = 0; j < R; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
         }
         __syncthreads();
     }
@@ -93,12 +107,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
     const float* bias = g.bias ? g.bias + (size_t)z * g.sBiasz : nullptr;
     const float* mask = g.mask ? g.mask + (size_t)z * g.sMz : nullptr;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int m = m0 + ty * 4 + i;
+    for (int i = 0; i < R; ++i) {
+        const int m = m0 + ty * R + i;
         if (m >= g.M) continue;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int n = n0 + tx * 4 + j;
+        for (int j = 0; j < R; ++j) {
+            const int n = n0 + tx * R + j;
             if (n >= g.N) continue;
             float v = acc[i][j];
             if (bias) v += bias[n];
@@ -157,9 +171,15 @@ __global__ void bias_grad_kernel(int B, int out_dim, const float* __restrict__ d
     G[(size_t)i * ld + b_off + o] = s;
 }
 
-int run_gemm(const GemmArgs& g, int batch, cudaStream_t s) {
-    dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, batch);
-    gemm_simt_kernel<<<grid, 256, 0, s>>>(g);
+int run_gemm(const GemmArgs& g, int batch, int sm_count, cudaStream_t s) {
+    const long long big = (long long)((g.N + 63) / 64) * ((g.M + 63) / 64) * batch;
+    if (big >= 4LL * sm_count) {
+        dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, batch);
+        gemm_simt_kernel<4><<<grid, 256, 0, s>>>(g);
+    } else {
+        dim3 grid((g.N + 31) / 32, (g.M + 31) / 32, batch);
+        gemm_simt_kernel<2><<<grid, 256, 0, s>>>(g);
+    }
     DBW_LAUNCHED();
     return DBW_OK;
 }
@@ -204,7 +224,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.C = h->d_act[l + 1]; g.sCz = (long long)B * out; g.sCm = out;
         g.bias = X + m.b_off[l]; g.sBiasz = h->ld;
         g.M = B; g.N = out; g.K = in; g.relu = l < L - 1;
-        if ((rc = run_gemm(g, N, s)) != DBW_OK) return rc;
+        if ((rc = run_gemm(g, N, h->sm_count, s)) != DBW_OK) return rc;
     }
     softmax_ce_kernel<<<N, 256, 0, s>>>(B, m.dims[L], h->d_act[L], h->d_ylab, h->d_dz[L], loss);
     DBW_LAUNCHED();
@@ -216,7 +236,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.B = h->d_act[l]; g.sBz = (long long)B * in; g.sBn = 1; g.sBk = in;
         g.C = G + m.w_off[l]; g.sCz = h->ld; g.sCm = in;
         g.M = out; g.N = in; g.K = B;
-        if ((rc = run_gemm(g, N, s)) != DBW_OK) return rc;
+        if ((rc = run_gemm(g, N, h->sm_count, s)) != DBW_OK) return rc;
         bias_grad_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(B, out, h->d_dz[l + 1], G, h->ld, m.b_off[l]);
         DBW_LAUNCHED();
         if (l > 0) {  // dZ_{l}[m][k] = (sum_o dZ_{l+1}[m][o] W_l[o][k]) * [A_l[m][k] > 0]
@@ -226,7 +246,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
             a.C = h->d_dz[l]; a.sCz = (long long)B * in; a.sCm = in;
             a.mask = h->d_act[l]; a.sMz = (long long)B * in; a.sMm = in;
             a.M = B; a.N = in; a.K = out;
-            if ((rc = run_gemm(a, N, s)) != DBW_OK) return rc;
+            if ((rc = run_gemm(a, N, h->sm_count, s)) != DBW_OK) return rc;
         }
     }
     return DBW_OK;
