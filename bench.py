@@ -358,14 +358,44 @@ def run_ours(args):
         overrides["samples"] = args.samples
     if args.width:
         overrides["d"] = args.width
-    job = Job(args.config, device=local, **overrides)
-    w = job.w
-    for _ in range(args.warmup):
-        job.step()
-    torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    res = measure(args.config, local, args, dist, overrides)
+    extra = {}
+    # the whole hot path with a model (gradients on the tensor cores) next to the mix-only headline
+    also = [c for c in (args.also or []) if c != args.config] if world == 1 and not overrides else []
+    for c in also:
+        extra[wl.CONFIGS[c]["name"]] = summary(measure(c, local, args, dist, {}), world, args)
+    clocks = sampler.stop() if rank == 0 else None
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    w = res["w"]
+    line = {"metric": METRIC, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic"}
+    line.update(summary(res, world, args))
+    line["roofline"]["traffic"] = MIX_TRAFFIC_BYTES.get(args.config) if not overrides else None
+    line["clocks"] = clocks
+    if extra:
+        line["other_workloads"] = extra
+    if not args.no_cpu_baseline and world == 1:
+        sec, desc = oracle_sample_seconds(w, 0, budget_s=args.ref_budget)
+        line["cpu_baseline"] = {"value": w.N / sec, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def measure(config, local, args, dist, overrides):
+    """Device-resident loop, stage times, launch count and the end-to-end loop of one workload."""
+    import torch
+    from paper_2102_06280_b200 import binding
+    job = Job(config, device=local, **overrides)
+    for _ in range(args.warmup):
+        job.step()
+    torch.cuda.synchronize()
     job.h.profile(True)
     job.h.profile_read()
     launches0 = binding.launch_count()
@@ -377,45 +407,54 @@ def run_ours(args):
     for _ in range(min(args.warmup, 3)):
         job.step_host()
     ms_e2e = timed_loop(job, args.steps, job.step_host, dist)
-    clocks = sampler.stop() if rank == 0 else None
-    status = job.h.status()
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
-    peaks, peak_kind = measured_peaks()
-    value = aggregate_value(w.N, args.steps, ms, world)
-    e2e = aggregate_value(w.N, args.steps, ms_e2e, world)
-    h2d, d2h = job.host_bytes_per_step()
-    mix_ms = stage_ms["mix"] / max(stage_rounds, 1)
-    achieved = job.mix_bytes_per_launch() / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
-    staged = w.weight_rule == "uniform" and 64 <= w.N <= 1024 and w.N * 128 > 113 * 1024
-    roofline = {"kernel": "mix_staged_kernel" if staged else "mix_panel_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind,
-                "frac_of_8TBps_nominal": achieved / 8000.0,
-                "traffic": MIX_TRAFFIC_BYTES.get(args.config) if not (args.width or args.samples) else None,
-                "bytes_per_launch": job.mix_bytes_per_launch(), "ms_per_launch": mix_ms}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32" if w.precision == "fp32" else "bf16xbf16->f32 GEMM, f32 mix",
-            "data": "synthetic",
-            "config": {"workload": w.name, "N": w.N, "d": w.d, "ld": job.ld, "nnz": int(len(w.col)),
-                       "batch": w.batch, "layers": w.layers, "backups": w.backups, "weights": w.weight_rule,
-                       "l2": "inputs larger than L2 (X and G each %.2f GB)" % (w.N * job.ld * 4 / 1e9)
-                             if w.N * job.ld * 4 > 126e6 else "working set smaller than L2: cache-resident by design",
-                       "multi_gpu": "replicas only" if world > 1 else "single GPU"},
-            "stage_ms": {k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
-            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": ms_e2e / args.steps},
-            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks, "device_status": status}
-    if not args.no_cpu_baseline and world == 1:
-        sec, desc = oracle_sample_seconds(w, 0, budget_s=args.ref_budget)
-        line["cpu_baseline"] = {"value": w.N / sec, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc}
-    print(json.dumps(line))
+    out = dict(w=job.w, ld=job.ld, ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
+               stage_ms={k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
+               bytes=job.host_bytes_per_step(), mix_bytes=job.mix_bytes_per_launch())
     job.close()
-    if dist is not None:
-        dist.destroy_process_group()
+    del job
+    torch.cuda.empty_cache()
+    return out
+
+
+def model_flops_per_round(w):
+    """Dense-layer flops of one round: forward + dW (2 each per weight and sample) + dA for layers above the first."""
+    if w.layers is None:
+        return 0
+    dims = wl.layer_dims(w.layers)
+    per_sample = sum(4 * o * i for o, i in dims) + sum(2 * o * i for o, i in dims[1:])
+    return per_sample * w.batch * w.N
+
+
+def summary(res, world, args):
+    w = res["w"]
+    peaks, peak_kind = measured_peaks()
+    mix_ms = res["stage_ms"]["mix"]
+    achieved = res["mix_bytes"] / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
+    staged = w.weight_rule == "uniform" and 64 <= w.N <= 1024 and w.N * 128 > 113 * 1024
+    h2d, d2h = res["bytes"]
+    out = {"value": aggregate_value(w.N, args.steps, res["ms"], world), "ms_per_step": res["ms"] / args.steps,
+           "dtype": "f32" if w.precision == "fp32" else "bf16",
+           "config": {"workload": w.name, "N": w.N, "d": w.d, "ld": res["ld"], "nnz": int(len(w.col)),
+                      "batch": w.batch, "layers": w.layers, "backups": w.backups, "weights": w.weight_rule,
+                      "precision": "fp32" if w.precision == "fp32" else "bf16 operands, fp32 accumulate, fp32 master and mix",
+                      "l2": "inputs larger than L2 (X and G each %.2f GB)" % (w.N * res["ld"] * 4 / 1e9)
+                            if w.N * res["ld"] * 4 > 126e6 else "working set smaller than L2: cache-resident by design",
+                      "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+           "stage_ms": res["stage_ms"],
+           "e2e": {"value": aggregate_value(w.N, args.steps, res["ms_e2e"], world), "unit": UNIT,
+                   "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": res["ms_e2e"] / args.steps},
+           "gpu_launches": int(res["launches"]),
+           "roofline": {"kernel": "mix_staged_kernel" if staged else "mix_panel_kernel", "bound": "hbm",
+                        "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                        "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
+                        "bytes_per_launch": res["mix_bytes"], "ms_per_launch": mix_ms},
+           "device_status": res["status"]}
+    flops = model_flops_per_round(w)
+    if flops and res["stage_ms"]["grad"] > 0:
+        out["gradients"] = {"dense_flop_per_round": flops,
+                            "tflops_over_grad_stage": flops / (res["stage_ms"]["grad"] * 1e-3) / 1e12,
+                            "note": "grad stage = gather, casts, GEMMs, loss and last layer together"}
+    return out
 
 
 def main():
@@ -427,6 +466,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU oracle work per sampled step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--also", type=int, nargs="*", default=[3], choices=sorted(wl.CONFIGS),
+                    help="further workloads summarised under other_workloads (single GPU only)")
     ap.add_argument("--samples", type=int, default=0, help="profiling aid: samples per worker instead of the config's")
     ap.add_argument("--width", type=int, default=0, help="profiling aid: columns d of the mix-only config instead of 2^20")
     args = ap.parse_args()
