@@ -284,3 +284,46 @@ def test_grad_bf16_tensor_cores_match_oracle(dims, batch, n):
         assert abs(float(loss[i]) - l) <= 2e-2 * max(abs(l), 1.0)
     assert np.count_nonzero(G.cpu().numpy()) <= m.d * n     # padding untouched
     h.close()
+
+
+def test_degenerate_sizes():
+    """One worker (no links), two workers, and a padded leading dimension far above d."""
+    p = _dbw()
+    # N = 1: no neighbours, the round is a plain SGD step and lasts t_0
+    rowptr, col = np.array([0, 0], dtype=np.int32), np.zeros(0, dtype=np.int32)
+    h = p.Dbw(rowptr, col, d=10, ld=12)
+    X = torch.arange(12, dtype=torch.float32, device="cuda").reshape(1, 12)
+    G = torch.ones(1, 12, device="cuda")
+    kept = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    Tw = torch.zeros(1, dtype=torch.float64, device="cuda")
+    Tr = torch.zeros(1, dtype=torch.float64, device="cuda")
+    out = torch.empty_like(X)
+    t, b = dev(np.array([2.5])), dev(np.zeros(1, dtype=np.int32))
+    h.round(X, t, b, 0.5, out, kept, G_ext=G, T_worker=Tw, T_round=Tr)
+    torch.cuda.synchronize()
+    assert torch.equal(out, X - 0.5 * G)
+    assert float(Tw[0]) == 0.0 and float(Tr[0]) == 0.0         # nobody waits for anybody: no participant
+    bo = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    th = torch.zeros(1, dtype=torch.float64, device="cuda")
+    h.update_backups(t, bo, th)                                   # no links: threshold +inf, b = deg = 0
+    torch.cuda.synchronize()
+    assert int(bo[0]) == 0 and np.isinf(float(th[0]))
+    assert h.status() == 0
+    h.close()
+    # N = 2, ld much larger than d (the tail is padding and must stay zero)
+    rowptr, col = wl.path(2)
+    d, ld = 6, 512
+    h = p.Dbw(rowptr, col, d=d, ld=ld)
+    rng = np.random.default_rng(0)
+    Xh = np.zeros((2, ld), dtype=np.float32); Gh = np.zeros((2, ld), dtype=np.float32)
+    Xh[:, :d] = rng.standard_normal((2, d)); Gh[:, :d] = rng.standard_normal((2, d))
+    Xd = dev(Xh)
+    kept = torch.zeros(2, dtype=torch.uint8, device="cuda")
+    tt, bb = np.array([1.0, 1.0]), np.zeros(2, dtype=np.int32)
+    h.round(Xd, dev(tt), dev(bb), 0.1, Xd, kept, G_ext=dev(Gh))
+    torch.cuda.synchronize()
+    r = orc.dbw_round(rowptr, col, Xh, tt, bb, 0.1, G=Gh)
+    assert row_rel_err(Xd.cpu().numpy()[:, :d], r["X"][:, :d]) <= 1e-5
+    assert not np.any(Xd.cpu().numpy()[:, d:])
+    assert np.array_equal(kept.cpu().numpy(), r["kept"])
+    h.close()
