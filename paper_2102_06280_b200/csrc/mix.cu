@@ -25,7 +25,7 @@ __device__ __forceinline__ float4 fma4(float w, float4 v, float4 a) {
 }
 
 template <int GS>
-__global__ void __launch_bounds__(kMixThreads)
+__global__ void __launch_bounds__(kMixThreads, 3)
 mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ G, float lr,
                  const float* __restrict__ lr_pw, float* Xout, uint16_t* __restrict__ shadow, MixPlan plan,
                  int mix_then_correct, int n_panels) {
