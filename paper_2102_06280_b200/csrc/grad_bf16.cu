@@ -6,9 +6,10 @@
 //   dA_l            = dZ_{l+1} W_l         A-operand dZ_{l+1} [B][out]   B-operand W_l^T      [in][out]
 // so every producer of an activation or of a dZ also writes its transpose.  Tiles are staged by
 // TMA (3-D maps: K, rows, worker; 128-byte swizzle; no multicast) through an mbarrier ring, one
-// elected thread issues tcgen05.mma, and four warps drain the accumulator with tcgen05.ld into the
-// fused epilogues (bias + ReLU + bf16 cast, ReLU mask, or fp32 straight into G).  The last layer
-// (a handful of classes) and the loss run on the CUDA cores from the fp32 master weights.
+// elected thread issues tcgen05.mma into one of two accumulator buffers in tensor memory, and eight
+// warps drain the finished buffer with tcgen05.ld into the fused epilogues (bias + ReLU + bf16
+// cast, ReLU mask, or fp32 straight into G) while the next tile is already being multiplied.  The
+// last layer (a handful of classes) and the loss run on the CUDA cores from the fp32 master weights.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
