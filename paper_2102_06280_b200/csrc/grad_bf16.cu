@@ -13,6 +13,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -488,21 +489,22 @@ __global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, floa
 template <int CP, int KPT>
 __global__ void __launch_bounds__(64)
 head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld,
-                     long long w_off, long long b_off, const float* __restrict__ dzL, float* __restrict__ G,
+                     long long w_off, const float* __restrict__ dzL, float* __restrict__ G, float* __restrict__ dwp,
                      bf16* __restrict__ dzP, bf16* __restrict__ dzPT) {
-    extern __shared__ float4 sdz4[];  // [B][CP] floats
+    // blockIdx.z splits the batch (in chunks of 8 samples) so that enough blocks are in flight; with
+    // more than one part the dW partial sums go to dwp [part][worker][C][K] and head_reduce_kernel
+    // adds them in a fixed order.
+    extern __shared__ float4 sdz4[];  // [samples of this part][CP] floats
     float* sdz = reinterpret_cast<float*>(sdz4);
     const int i = blockIdx.y;
-    for (int e = threadIdx.x; e < B * CP; e += blockDim.x) {
-        const int s = e / CP, c = e % CP;
+    const int nch = B / 8;
+    const int s_lo = 8 * (int)((long long)blockIdx.z * nch / gridDim.z);
+    const int s_hi = 8 * (int)((long long)(blockIdx.z + 1) * nch / gridDim.z);
+    for (int e = threadIdx.x; e < (s_hi - s_lo) * CP; e += blockDim.x) {
+        const int s = s_lo + e / CP, c = e % CP;
         sdz[e] = c < C ? dzL[((size_t)i * B + s) * C + c] : 0.f;
     }
     __syncthreads();
-    if (blockIdx.x == 0 && threadIdx.x < C) {
-        float t = 0.f;
-        for (int s = 0; s < B; ++s) t += sdz[s * CP + threadIdx.x];
-        G[(size_t)i * ld + b_off + threadIdx.x] = t;
-    }
     const int k = (blockIdx.x * 64 + threadIdx.x) * KPT;
     if (k >= K) return;  // K % 8 == 0, so k + KPT <= K
     float w[CP][KPT], dw[CP][KPT];
@@ -518,7 +520,7 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             raw[u] = 0u;
-            if (s0 + u < B) {
+            if (s0 + u < s_hi) {
                 if (KPT == 2)
                     raw[u] = __ldg(reinterpret_cast<const uint32_t*>(a + (size_t)(s0 + u) * K));
                 else
@@ -527,8 +529,8 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
         }
     };
     uint32_t cur[8], nxt[8];
-    load_a(0, cur);
-    for (int s0 = 0; s0 < B; s0 += 8) {  // B % 8 == 0
+    load_a(s_lo, cur);
+    for (int s0 = s_lo; s0 < s_hi; s0 += 8) {  // B % 8 == 0
         load_a(s0 + 8, nxt);  // next eight samples in flight while these are used
         float dav[KPT][8];
 #pragma unroll
@@ -546,7 +548,7 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
             for (int q = 0; q < KPT; ++q) da[q] = 0.f;
 #pragma unroll
             for (int c4 = 0; c4 < CP / 4; ++c4) {
-                const float4 d4 = sdz4[s * (CP / 4) + c4];
+                const float4 d4 = sdz4[(s - s_lo) * (CP / 4) + c4];
                 const float dz[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
@@ -574,11 +576,30 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
 #pragma unroll
         for (int u = 0; u < 8; ++u) cur[u] = nxt[u];
     }
+    float* dst = gridDim.z == 1 ? G + (size_t)i * ld + w_off : dwp + ((size_t)blockIdx.z * gridDim.y + i) * C * K;
 #pragma unroll
     for (int c = 0; c < CP; ++c)
         if (c < C)
 #pragma unroll
-            for (int q = 0; q < KPT; ++q) G[(size_t)i * ld + w_off + (size_t)c * K + k + q] = dw[c][q];
+            for (int q = 0; q < KPT; ++q) dst[(size_t)c * K + k + q] = dw[c][q];
+}
+
+// dW of the last layer = sum of the batch parts' partial sums (fixed order), and db[c] = sum_s dZ[s][c].
+__global__ void __launch_bounds__(256)
+head_reduce_kernel(int B, int K, int C, int parts, int workers, const float* __restrict__ dwp, const float* __restrict__ dzL,
+                   float* __restrict__ G, long long ld, long long w_off, long long b_off) {
+    const int i = blockIdx.y;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (parts > 1 && e < C * K) {
+        float t = 0.f;
+        for (int z = 0; z < parts; ++z) t += dwp[((size_t)z * workers + i) * C * K + e];
+        G[(size_t)i * ld + w_off + e] = t;
+    }
+    if (e < C) {
+        float t = 0.f;
+        for (int s = 0; s < B; ++s) t += dzL[((size_t)i * B + s) * C + e];
+        G[(size_t)i * ld + b_off + e] = t;
+    }
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -625,6 +646,7 @@ struct BF16State {
     bf16* dZ[DBW_MAX_LAYERS] = {};   // dZ_l  [N][B][dims[l]],  l = 1..L-1
     bf16* dZT[DBW_MAX_LAYERS] = {};  // dZ_l^T
     float* dzL = nullptr;            // [N][B][C]
+    float* dwp = nullptr;            // [4][N][C][K_last] partial dW of the last layer
     float* loss_s = nullptr;         // [N][B]
     int32_t* ylab = nullptr;         // [N][B]
     CUtensorMap fwdA[DBW_MAX_LAYERS], fwdB[DBW_MAX_LAYERS], dwA[DBW_MAX_LAYERS], dwB[DBW_MAX_LAYERS],
@@ -688,6 +710,7 @@ int grad_bf16_alloc(dbw_handle* h) {
     ok = ok && balloc(st, &shadow, (size_t)N * h->ld);
     h->d_shadow = reinterpret_cast<uint16_t*>(shadow);
     for (int l = 0; l <= L - 2 && ok; ++l) st->Wh[l] = shadow + m.w_off[l];
+    ok = ok && balloc(st, &st->dwp, (size_t)4 * N * m.dims[L] * m.dims[L - 1]);
     ok = ok && balloc(st, &st->dzL, NB * m.dims[L]) && balloc(st, &st->loss_s, NB) && balloc(st, &st->ylab, NB);
     if (!ok) return DBW_ERR_CUDA;
     for (int l = 0; l <= L - 2; ++l) {
@@ -766,12 +789,16 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     }
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
     bf16* dzPT = L >= 2 ? st->dZT[L - 1] : nullptr;
+    const int parts = B >= 64 ? 4 : 1;
     if (C <= 16)
-        head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N), 64, (size_t)B * 16 * 4, s>>>(
-            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
+        head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP, dzPT);
     else
-        head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N), 64, (size_t)B * 32 * 4, s>>>(
-            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1], st->dzL, G, dzP, dzPT);
+        head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N, parts), 64, (size_t)B * 32 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP, dzPT);
+    DBW_LAUNCHED();
+    head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
+                                                                              m.w_off[L - 1], m.b_off[L - 1]);
     DBW_LAUNCHED();
     // backward through the tensor-core layers
     for (int l = L - 2; l >= 0; --l) {
