@@ -394,32 +394,32 @@ bias_grad_t_kernel(int out_dim, int B, const bf16* __restrict__ dzT, long long d
 constexpr int kMaxClasses = 32;
 
 // logits = A W^T + b (A bf16 [B][K], W fp32 master [C][K]), then dZ = (softmax - onehot)/B and the
-// per-sample loss.  A warp takes four samples at once: each lane owns 8 consecutive k of every
+// per-sample loss.  A warp takes HS samples at once: each lane owns 8 consecutive k of every
 // 256-wide chunk (one 128-bit load per sample, two per weight row), so a weight row fetched from
-// L1/L2 is used for four samples.
-template <int CP>
+// L1/L2 is used for HS samples.
+template <int CP, int HS>
 __global__ void __launch_bounds__(128)
 head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld, long long w_off,
                     long long b_off, const int32_t* __restrict__ ylab, float* __restrict__ dzL, float* __restrict__ loss_s) {
     const int i = blockIdx.y;
-    const int s0 = (blockIdx.x * 4 + (threadIdx.x >> 5)) * 4;
+    const int s0 = (blockIdx.x * 4 + (threadIdx.x >> 5)) * HS;
     const int lane = threadIdx.x & 31;
     if (s0 >= B) return;
     const float* W = X + (size_t)i * ld + w_off;
-    float acc[4][CP];
+    float acc[HS][CP];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < HS; ++u)
 #pragma unroll
         for (int c = 0; c < CP; ++c) acc[u][c] = 0.f;
-    auto load_a = [&](int kc, uint4 (&raw)[4]) {
+    auto load_a = [&](int kc, uint4 (&raw)[HS]) {
         const int k = kc + lane * 8;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < HS; ++u) {
             raw[u] = make_uint4(0u, 0u, 0u, 0u);
             if (k < K && s0 + u < B) raw[u] = __ldg(reinterpret_cast<const uint4*>(A + ((size_t)i * B + s0 + u) * K + k));
         }
     };
-    uint4 cur[4], nxt[4];
+    uint4 cur[HS], nxt[HS];
     load_a(0, cur);
     for (int kc = 0; kc < K; kc += 256) {
         load_a(kc + 256, nxt);  // next chunk in flight while this one is used (all zero past the end)
@@ -432,7 +432,7 @@ head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float
                     const float4 w1 = __ldg(reinterpret_cast<const float4*>(W + (size_t)c * K + k + 4));
                     const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < HS; ++u) {
                         const uint32_t w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {  // bf16 -> fp32 is a 16-bit shift
@@ -444,10 +444,10 @@ head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) cur[u] = nxt[u];
+        for (int u = 0; u < HS; ++u) cur[u] = nxt[u];
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < HS; ++u) {
         float z_mine = 0.f;  // lane c ends up holding logit c of sample s0 + u
 #pragma unroll
         for (int c = 0; c < CP; ++c) {
@@ -777,10 +777,10 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
     if (C <= 16)
-        head_forward_kernel<16><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+        head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     else
-        head_forward_kernel<32><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+        head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     DBW_LAUNCHED();
     if (loss) {
