@@ -1,11 +1,12 @@
 // Mini-batch stochastic gradient (Eq. 2) with the dense layers on the 5th-generation tensor cores:
 // BF16 operands (activations, and weights cast from the fp32 master rows every round), fp32
-// accumulation in tensor memory, fp32 gradients.  All GEMMs are "both operands K-major":
-//   forward   Z_{l+1} = A_l W_l^T          A-operand A_l      [B][in]    B-operand W_l        [out][in]
-//   dW_l            = dZ_{l+1}^T A_l       A-operand dZ_{l+1}^T [out][B]  B-operand A_l^T      [in][B]
-//   dA_l            = dZ_{l+1} W_l         A-operand dZ_{l+1} [B][out]   B-operand W_l^T      [in][out]
-// so every producer of an activation or of a dZ also writes its transpose.  Tiles are staged by
-// TMA (3-D maps: K, rows, worker; 128-byte swizzle; no multicast) through an mbarrier ring, one
+// accumulation in tensor memory, fp32 gradients.  No operand is ever transposed in memory: the MMA
+// reads an operand either K-major (the reduction index contiguous) or MN-major (the row / column
+// index contiguous), chosen per GEMM:
+//   forward   Z_{l+1} = A_l W_l^T       A: A_l      [B][in]   K-major    B: W_l      [out][in]  K-major
+//   dW_l            = dZ_{l+1}^T A_l    A: dZ_{l+1} [B][out]  MN-major   B: A_l      [B][in]    MN-major
+//   dA_l            = dZ_{l+1} W_l      A: dZ_{l+1} [B][out]  K-major    B: W_l      [out][in]  MN-major
+// Tiles are staged by TMA (3-D maps; 128-byte swizzle; no multicast) through an mbarrier ring, one
 // elected thread issues tcgen05.mma into one of two accumulator buffers in tensor memory, and eight
 // warps drain the finished buffer with tcgen05.ld into the fused epilogues (bias + ReLU + bf16
 // cast, ReLU mask, or fp32 straight into G) while the next tile is already being multiplied.  The
@@ -98,6 +99,20 @@ __device__ __forceinline__ uint64_t kmajor_sw128_desc(uint32_t smem_addr) {
     return d;
 }
 
+// MN-major tile (the M or N index is contiguous in memory, K runs over rows) staged by TMA in
+// chunks of 64 (MN) x 64 (K rows) with the 128-byte swizzle: inside a chunk a K row is 128 bytes,
+// groups of 8 K rows are 1024 bytes apart (stride byte offset); chunks along MN follow each other
+// 8192 bytes apart (leading byte offset).
+__device__ __forceinline__ uint64_t mnmajor_sw128_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(8192 >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
 // two floats -> packed bf16x2 (low half = first)
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -113,8 +128,11 @@ constexpr int EPI_WARPS = 8;
 constexpr size_t gemm_smem(int stages, int bn) {
     return (size_t)stages * (TILE_BYTES + bn * BK * 2) + 8 * 32 * 36 * 4 /*epilogue staging*/ + 1024 /*align slack*/ + 256 /*barriers*/;
 }
-// kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = bn
-__host__ __device__ constexpr uint32_t idesc_for(int bn) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24); }
+// kind::f16, D = f32, A = B = bf16, M = 128, N = bn; bits 15 / 16 select MN-major A / B operands
+__host__ __device__ constexpr uint32_t idesc_for(int bn, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(bn >> 3) << 17) |
+           ((uint32_t)(BM >> 4) << 24);
+}
 
 enum { EPI_FWD = 0, EPI_DA = 1, EPI_DW = 2 };
 
@@ -138,14 +156,14 @@ constexpr int STAGING_FLOATS = EPI_WARPS * 32 * 36;  // per epilogue warp a 32 x
 // Warp 0 streams operand tiles by TMA through a STAGES-deep ring, warp 1 issues the MMAs into one of
 // ACC accumulator buffers in tensor memory, warps 2-9 drain a finished buffer through the epilogue
 // while the next tile's loads and MMAs are already running.
-template <int STAGES, int BN, int ACC>
+template <int STAGES, int BN, int ACC, bool AMN, bool BMN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs g, int tiles_m,
                int tiles_n, int n_tiles) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int TILE_B_BYTES = BN * BK * 2;
-    constexpr uint32_t IDESC = idesc_for(BN);
+    constexpr uint32_t IDESC = idesc_for(BN, AMN, BMN);
     uint8_t* tilesA = smem;
     uint8_t* tilesB = smem + STAGES * TILE_BYTES;
     float* staging = reinterpret_cast<float*>(smem + STAGES * (TILE_BYTES + TILE_B_BYTES));
@@ -187,8 +205,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int s = it % STAGES;
                     if (it >= STAGES) mbar_wait(&empty[s], ((it / STAGES) - 1) & 1, g.status);
                     mbar_expect_tx(&full[s], TILE_BYTES + TILE_B_BYTES);
-                    tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
-                    tma_load_3d(tilesB + s * TILE_B_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+                    if (!AMN) {
+                        tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < BM / 64; ++c)  // MN-major: 64 x 64 chunks, coordinates (mn, k row, worker)
+                            tma_load_3d(tilesA + s * TILE_BYTES + c * 8192, &tmA, m0 + c * 64, kb * BK, z, &full[s]);
+                    }
+                    if (!BMN) {
+                        tma_load_3d(tilesB + s * TILE_B_BYTES, &tmB, kb * BK, n0, z, &full[s]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < BN / 64; ++c)
+                            tma_load_3d(tilesB + s * TILE_B_BYTES + c * 8192, &tmB, n0 + c * 64, kb * BK, z, &full[s]);
+                    }
                 }
             }
         }
@@ -206,12 +236,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int s = it % STAGES;
                     mbar_wait(&full[s], (it / STAGES) & 1, g.status);
                     tc_fence_after();
-                    const uint64_t da = kmajor_sw128_desc(smem_u32(tilesA + s * TILE_BYTES));
-                    const uint64_t db = kmajor_sw128_desc(smem_u32(tilesB + s * TILE_B_BYTES));
+                    const uint32_t sa = smem_u32(tilesA + s * TILE_BYTES), sb = smem_u32(tilesB + s * TILE_B_BYTES);
+                    const uint64_t da = AMN ? mnmajor_sw128_desc(sa) : kmajor_sw128_desc(sa);
+                    const uint64_t db = BMN ? mnmajor_sw128_desc(sb) : kmajor_sw128_desc(sb);
+                    // 16 further along K: 32 bytes inside the swizzle atom (K-major) or 16 rows of 128 bytes (MN-major)
+                    constexpr uint64_t ka = (AMN ? UMMA_K * 128 : UMMA_K * 2) / 16, kbs = (BMN ? UMMA_K * 128 : UMMA_K * 2) / 16;
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes further along K inside the swizzle atom
-                        tc_mma_bf16(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
-                                    (kb > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        tc_mma_bf16(d_tmem, da + (uint64_t)k * ka, db + (uint64_t)k * kbs, IDESC, (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit(&empty[s]);  // frees the stage once these MMAs have read it
                 }
                 tc_commit(&acc_full[buf]);
@@ -374,20 +406,18 @@ __global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ l
     }
 }
 
-// db[o] = sum over the batch of dZ[.][o], read from the transposed copy dZ^T [out][B]; warp per row.
+// db[o] = sum over the batch of dZ[s][o] (dZ bf16 [B][out]); thread per output, coalesced across o.
 __global__ void __launch_bounds__(128)
-bias_grad_t_kernel(int out_dim, int B, const bf16* __restrict__ dzT, long long dzT_z, float* __restrict__ G, long long ld,
-                   long long b_off) {
+bias_grad_bf16_kernel(int out_dim, int B, const bf16* __restrict__ dz, long long dz_z, float* __restrict__ G, long long ld,
+                      long long b_off) {
     const int i = blockIdx.y;
-    const int o = blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
     if (o >= out_dim) return;
-    const bf16* p = dzT + (size_t)i * dzT_z + (size_t)o * B;
+    const bf16* p = dz + (size_t)i * dz_z + o;
     float s = 0.f;
-    for (int m = lane; m < B; m += 32) s += __bfloat162float(p[m]);
-#pragma unroll
-    for (int k = 16; k > 0; k >>= 1) s += __shfl_xor_sync(0xffffffffu, s, k);
-    if (lane == 0) G[(size_t)i * ld + b_off + o] = s;
+#pragma unroll 8
+    for (int m = 0; m < B; ++m) s += __bfloat162float(p[(size_t)m * out_dim]);
+    G[(size_t)i * ld + b_off + o] = s;
 }
 
 // ----------------------------------------------------------------------------- last layer on CUDA cores
@@ -620,6 +650,20 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// MN-major operand [workers][K rows][MN] bf16 (MN contiguous): box = 64 (MN) x 64 (K rows) x 1.
+bool make_operand_map_mn(CUtensorMap* map, const bf16* base, int MN, int Krows, int workers, long long worker_pitch = 0) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    if (!worker_pitch) worker_pitch = (long long)MN * Krows;
+    cuuint64_t dims[3] = {(cuuint64_t)MN, (cuuint64_t)Krows, (cuuint64_t)workers};
+    cuuint64_t strides[2] = {(cuuint64_t)MN * 2, (cuuint64_t)worker_pitch * 2};
+    cuuint32_t box[3] = {64, 64, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // K-major operand [workers][rows][K] bf16: box = 64 (K) x 128 (rows) x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
 bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers, long long worker_pitch = 0,
@@ -640,11 +684,8 @@ bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int w
 
 struct BF16State {
     bf16* A[DBW_MAX_LAYERS] = {};    // A_l   [N][B][dims[l]],  l = 0..L-1
-    bf16* AT[DBW_MAX_LAYERS] = {};   // A_l^T [N][dims[l]][B],  l = 0..L-2
     bf16* Wh[DBW_MAX_LAYERS] = {};   // W_l   [out][in] inside the bf16 shadow rows (worker pitch ld), l = 0..L-2
-    bf16* WhT[DBW_MAX_LAYERS] = {};  // W_l^T [N][in][out],     l = 1..L-2
     bf16* dZ[DBW_MAX_LAYERS] = {};   // dZ_l  [N][B][dims[l]],  l = 1..L-1
-    bf16* dZT[DBW_MAX_LAYERS] = {};  // dZ_l^T
     float* dzL = nullptr;            // [N][B][C]
     float* dwp = nullptr;            // [4][N][C][K_last] partial dW of the last layer
     float* loss_s = nullptr;         // [N][B]
@@ -667,17 +708,31 @@ int tile_bn(int N) { return N >= 256 ? 256 : 128; }
 
 int g_tc_sm_count = 0;
 
-int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
+template <bool AMN, bool BMN>
+int run_tc_major(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
     const int bn = tile_bn(g.N);
     const int tiles_n = (g.N + bn - 1) / bn, tiles_m = (g.M + BM - 1) / BM;
     const int n_tiles = tiles_n * tiles_m * workers;
     const int grid = n_tiles < g_tc_sm_count ? n_tiles : g_tc_sm_count;
+    static bool configured = false;
+    if (!configured) {
+        DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<4, 128, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(4, 128)));
+        DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 256, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 256)));
+        configured = true;
+    }
     if (bn == 128)
-        gemm_tc_kernel<4, 128, 2><<<grid, GEMM_THREADS, gemm_smem(4, 128), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
+        gemm_tc_kernel<4, 128, 2, AMN, BMN><<<grid, GEMM_THREADS, gemm_smem(4, 128), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
     else
-        gemm_tc_kernel<3, 256, 2><<<grid, GEMM_THREADS, gemm_smem(3, 256), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
+        gemm_tc_kernel<3, 256, 2, AMN, BMN><<<grid, GEMM_THREADS, gemm_smem(3, 256), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
     DBW_LAUNCHED();
     return DBW_OK;
+}
+
+int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s, bool a_mn = false,
+           bool b_mn = false) {
+    if (a_mn && b_mn) return run_tc_major<true, true>(a, b, g, workers, s);
+    if (b_mn) return run_tc_major<false, true>(a, b, g, workers, s);
+    return run_tc_major<false, false>(a, b, g, workers, s);
 }
 }  // namespace
 
@@ -698,12 +753,9 @@ int grad_bf16_alloc(dbw_handle* h) {
     for (int l = 0; l < L && ok; ++l) {
         ok = ok && balloc(st, &st->A[l], NB * m.dims[l]);
         if (l <= L - 2) {
-            ok = ok && balloc(st, &st->AT[l], NB * m.dims[l]);
-            if (l >= 1) ok = ok && balloc(st, &st->WhT[l], (size_t)N * m.dims[l] * m.dims[l + 1]);
         }
         if (l >= 1) {
             ok = ok && balloc(st, &st->dZ[l], NB * m.dims[l]);
-            ok = ok && balloc(st, &st->dZT[l], NB * m.dims[l]);
         }
     }
     bf16* shadow = nullptr;
@@ -716,17 +768,15 @@ int grad_bf16_alloc(dbw_handle* h) {
     for (int l = 0; l <= L - 2; ++l) {
         ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
         ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1]));
-        ok = ok && make_operand_map(&st->dwA[l], st->dZT[l + 1], B, m.dims[l + 1], N);
-        ok = ok && make_operand_map(&st->dwB[l], st->AT[l], B, m.dims[l], N, 0, tile_bn(m.dims[l]));
+        ok = ok && make_operand_map_mn(&st->dwA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
+        ok = ok && make_operand_map_mn(&st->dwB[l], st->A[l], m.dims[l], B, N);
         if (l >= 1) {
             ok = ok && make_operand_map(&st->daA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
-            ok = ok && make_operand_map(&st->daB[l], st->WhT[l], m.dims[l + 1], m.dims[l], N, 0, tile_bn(m.dims[l]));
+            ok = ok && make_operand_map_mn(&st->daB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld);
         }
     }
     if (!ok) return DBW_ERR_CUDA;
     g_tc_sm_count = h->sm_count;
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<4, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(4, 128)));
-    DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 256)));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
@@ -745,22 +795,19 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     BF16State* st = h->bf16;
     const int L = m.n_layers, B = m.batch, N = h->N, C = m.dims[L];
     int rc;
-    // bf16 copies of the weights of the tensor-core layers (inside the shadow rows) and their
-    // transposes for dA.  When the previous mix already wrote the shadow of this very X, only the
-    // transposes are left to do.
+    // bf16 copies of the weights of the tensor-core layers (inside the shadow rows), unless the
+    // previous mix already wrote the shadow of this very X.
     const bool have_shadow = h->track_params && h->shadow_valid && h->shadow_of == X;
-    for (int l = 0; l <= L - 2; ++l) {
+    for (int l = 0; l <= L - 2 && !have_shadow; ++l) {
         const int in = m.dims[l], out = m.dims[l + 1];
-        if (have_shadow && l == 0) continue;
         cast_tile_kernel<<<dim3((in + 63) / 64, (out + 63) / 64, N), 256, 0, s>>>(
-            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, have_shadow ? nullptr : st->Wh[l], h->ld,
-            l >= 1 ? st->WhT[l] : nullptr, (long long)in * out, h->d_status);
+            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], h->ld, nullptr, 0, h->d_status);
         DBW_LAUNCHED();
     }
-    // mini-batch gather: A_0 (and A_0^T when a tensor-core layer consumes it)
+    // mini-batch gather: A_0 in bf16
     cast_tile_kernel<<<dim3((m.dims[0] + 63) / 64, (B + 63) / 64, N), 256, 0, s>>>(
         B, m.dims[0], h->feat, (long long)h->S * m.dims[0], m.dims[0], batch_idx, B, h->S, st->A[0], (long long)B * m.dims[0],
-        L >= 2 ? st->AT[0] : nullptr, (long long)B * m.dims[0], h->d_status);
+        nullptr, 0, h->d_status);
     DBW_LAUNCHED();
     gather_labels_kernel<<<N, 128, 0, s>>>(B, h->S, h->labels, batch_idx, st->ylab);
     DBW_LAUNCHED();
@@ -769,7 +816,6 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         TcArgs g{};
         g.M = B; g.N = m.dims[l + 1]; g.K = m.dims[l]; g.epi = EPI_FWD;
         g.out = st->A[l + 1]; g.out_z = (long long)B * g.N; g.out_pitch = g.N;
-        g.outT = (l + 1 <= L - 2) ? st->AT[l + 1] : nullptr; g.outT_z = (long long)B * g.N; g.outT_pitch = B;
         g.bias = X + m.b_off[l]; g.bias_z = h->ld;
         g.status = h->d_status;
         if ((rc = run_tc(st->fwdA[l], st->fwdB[l], g, N, s))) return rc;
@@ -788,7 +834,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         DBW_LAUNCHED();
     }
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
-    bf16* dzPT = L >= 2 ? st->dZT[L - 1] : nullptr;
+    bf16* dzPT = nullptr;  // the dW GEMMs read dZ itself as an MN-major operand
     const int parts = B >= 64 ? 4 : 1;
     if (C <= 16)
         head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
@@ -807,17 +853,16 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         w.M = out; w.N = in; w.K = B; w.epi = EPI_DW;
         w.outf = G + m.w_off[l]; w.outf_z = h->ld; w.outf_pitch = in;
         w.status = h->d_status;
-        if ((rc = run_tc(st->dwA[l], st->dwB[l], w, N, s))) return rc;
-        bias_grad_t_kernel<<<dim3((out + 3) / 4, N), 128, 0, s>>>(out, B, st->dZT[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
+        if ((rc = run_tc(st->dwA[l], st->dwB[l], w, N, s, true, true))) return rc;
+        bias_grad_bf16_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(out, B, st->dZ[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
         DBW_LAUNCHED();
         if (l >= 1) {
             TcArgs a{};
             a.M = B; a.N = in; a.K = out; a.epi = EPI_DA;
             a.out = st->dZ[l]; a.out_z = (long long)B * in; a.out_pitch = in;
-            a.outT = st->dZT[l]; a.outT_z = (long long)B * in; a.outT_pitch = B;
             a.mask = st->A[l]; a.mask_z = (long long)B * in; a.mask_pitch = in;
             a.status = h->d_status;
-            if ((rc = run_tc(st->daA[l], st->daB[l], a, N, s))) return rc;
+            if ((rc = run_tc(st->daA[l], st->daB[l], a, N, s, false, true))) return rc;
         }
     }
     return DBW_OK;
