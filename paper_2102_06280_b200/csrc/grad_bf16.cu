@@ -139,7 +139,6 @@ enum { EPI_FWD = 0, EPI_DA = 1, EPI_DW = 2 };
 struct TcArgs {
     int M, N, K, epi;
     bf16* out;  long long out_z;  int out_pitch;    // [M][N] bf16 (EPI_FWD, EPI_DA)
-    bf16* outT; long long outT_z; int outT_pitch;   // [N][M] bf16, nullable
     float* outf; long long outf_z; long long outf_pitch;  // [M][N] fp32 (EPI_DW)
     const float* bias; long long bias_z;            // fp32 [N] (EPI_FWD)
     const bf16* mask; long long mask_z; int mask_pitch;   // bf16 [M][N]: keep where > 0 (EPI_DA)
@@ -316,12 +315,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int j = 0; j < 32; j += 8)
                         if (nb + j < g.N)
                             *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[j / 2], o[j / 2 + 1], o[j / 2 + 2], o[j / 2 + 3]);
-                    if (g.outT) {
-                        unsigned short* dt = reinterpret_cast<unsigned short*>(g.outT + (size_t)z * g.outT_z + (size_t)nb * g.outT_pitch + m);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < g.N) dt[(size_t)j * g.outT_pitch] = (unsigned short)((o[j >> 1] >> (16 * (j & 1))) & 0xffffu);
-                    }
                 }
             }
             // this warp's reads of the buffer are complete (tcgen05.wait::ld): hand it back to the MMA warp
@@ -339,11 +332,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ----------------------------------------------------------------------------- casts and gathers
-// fp32 [rows][cols] (row pitch src_pitch) -> bf16 [rows][cols] and, if dstT, bf16 [cols][rows].
-// Rows may be indirect (row_idx: mini-batch gather).  cols % 8 == 0 and rows % 8 == 0.
-// A block of 256 threads handles a 64 x 64 tile: every thread loads 16 consecutive floats of one
-// row (four 128-bit loads), stores them as 16 bf16 (two 128-bit stores), and for the transpose the
-// tile passes through shared memory so that the transposed rows leave as 128-bit stores too.
+// fp32 [rows][cols] (row pitch src_pitch) -> bf16 [rows][cols] (row pitch cols).  Rows may be
+// indirect (row_idx: mini-batch gather).  cols % 8 == 0.  Every thread converts 16 consecutive floats
+// of one row: four 128-bit loads, two 128-bit stores.
 __device__ __forceinline__ uint4 pack8(const float* v) {
     return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 }
@@ -351,49 +342,32 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
 __global__ void __launch_bounds__(256)
 cast_tile_kernel(int rows, int cols, const float* __restrict__ src, long long src_z, long long src_pitch,
                  const int32_t* __restrict__ row_idx, int idx_z, int idx_limit, bf16* __restrict__ dst, long long dst_z,
-                 bf16* __restrict__ dstT, long long dstT_z, uint32_t* status) {
-    __shared__ float tile[64][65];
+                 uint32_t* status) {
     const int z = blockIdx.z;
     const int t = threadIdx.x;
     const int r = blockIdx.y * 64 + (t >> 2);
     const int c0 = blockIdx.x * 64 + (t & 3) * 16;
+    if (r >= rows || c0 >= cols) return;
+    long long sr = r;
+    if (row_idx) {
+        int s = row_idx[(size_t)z * idx_z + r];
+        if (s < 0 || s >= idx_limit) {
+            atomicOr(status, DBW_STATUS_BAD_INDEX);
+            s = s < 0 ? 0 : idx_limit - 1;
+        }
+        sr = s;
+    }
+    const float* p = src + (size_t)z * src_z + sr * src_pitch + c0;
+    bf16* d = dst + (size_t)z * dst_z + (size_t)r * cols + c0;
     float v[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) v[e] = 0.f;
-    if (r < rows) {
-        long long sr = r;
-        if (row_idx) {
-            int s = row_idx[(size_t)z * idx_z + r];
-            if (s < 0 || s >= idx_limit) {
-                atomicOr(status, DBW_STATUS_BAD_INDEX);
-                s = s < 0 ? 0 : idx_limit - 1;
-            }
-            sr = s;
-        }
-        const float* p = src + (size_t)z * src_z + sr * src_pitch + c0;
-        bf16* d = dst + (size_t)z * dst_z + (size_t)r * cols + c0;
-#pragma unroll
-        for (int e = 0; e < 16; e += 4)
-            if (c0 + e < cols) {
-                const float4 f = __ldg(reinterpret_cast<const float4*>(p + e));
-                v[e] = f.x; v[e + 1] = f.y; v[e + 2] = f.z; v[e + 3] = f.w;
-            }
-        if (dst && c0 < cols) *reinterpret_cast<uint4*>(d) = pack8(v);
-        if (dst && c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
+    for (int e = 0; e < 16; e += 4) {
+        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c0 + e < cols) f = __ldg(reinterpret_cast<const float4*>(p + e));
+        v[e] = f.x; v[e + 1] = f.y; v[e + 2] = f.z; v[e + 3] = f.w;
     }
-    if (!dstT) return;
-#pragma unroll
-    for (int e = 0; e < 16; ++e) tile[t >> 2][(t & 3) * 16 + e] = v[e];
-    __syncthreads();
-    const int c = blockIdx.x * 64 + (t >> 2);
-    const int r0 = blockIdx.y * 64 + (t & 3) * 16;
-    if (c >= cols) return;
-    float w[16];
-#pragma unroll
-    for (int e = 0; e < 16; ++e) w[e] = tile[(t & 3) * 16 + e][t >> 2];
-    bf16* d = dstT + (size_t)z * dstT_z + (size_t)c * rows + r0;
-    if (r0 < rows) *reinterpret_cast<uint4*>(d) = pack8(w);
-    if (r0 + 8 < rows) *reinterpret_cast<uint4*>(d + 8) = pack8(w + 8);
+    *reinterpret_cast<uint4*>(d) = pack8(v);
+    if (c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
 }
 
 __global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
@@ -514,13 +488,13 @@ __global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, floa
 
 // Last layer backward; a thread owns KPT consecutive input features k:
 //   dW[c][k] = sum_s dZ[s][c] A[s][k],  db[c] = sum_s dZ[s][c],
-//   dZprev[s][k] = [A[s][k] > 0] * sum_c dZ[s][c] W[c][k]   (bf16, plus its transpose [K][B]).
+//   dZprev[s][k] = [A[s][k] > 0] * sum_c dZ[s][c] W[c][k]   (bf16).
 // dZ of the worker sits in shared memory and is read as 128-bit broadcasts.
 template <int CP, int KPT>
 __global__ void __launch_bounds__(64)
 head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld,
                      long long w_off, const float* __restrict__ dzL, float* __restrict__ G, float* __restrict__ dwp,
-                     bf16* __restrict__ dzP, bf16* __restrict__ dzPT) {
+                     bf16* __restrict__ dzP) {
     // blockIdx.z splits the batch (in chunks of 8 samples) so that enough blocks are in flight; with
     // more than one part the dW partial sums go to dwp [part][worker][C][K] and head_reduce_kernel
     // adds them in a fixed order.
@@ -597,12 +571,6 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
                     dzP[((size_t)i * B + s) * K + k] = __float2bfloat16_rn(dav[0][u]);
             }
         }
-        if (dzPT)
-#pragma unroll
-            for (int q = 0; q < KPT; ++q)
-                *reinterpret_cast<uint4*>(dzPT + ((size_t)i * K + k + q) * B + s0) =
-                    make_uint4(pack_bf16x2(dav[q][0], dav[q][1]), pack_bf16x2(dav[q][2], dav[q][3]),
-                               pack_bf16x2(dav[q][4], dav[q][5]), pack_bf16x2(dav[q][6], dav[q][7]));
 #pragma unroll
         for (int u = 0; u < 8; ++u) cur[u] = nxt[u];
     }
@@ -801,13 +769,13 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     for (int l = 0; l <= L - 2 && !have_shadow; ++l) {
         const int in = m.dims[l], out = m.dims[l + 1];
         cast_tile_kernel<<<dim3((in + 63) / 64, (out + 63) / 64, N), 256, 0, s>>>(
-            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], h->ld, nullptr, 0, h->d_status);
+            out, in, X + m.w_off[l], h->ld, in, nullptr, 0, 0, st->Wh[l], h->ld, h->d_status);
         DBW_LAUNCHED();
     }
     // mini-batch gather: A_0 in bf16
     cast_tile_kernel<<<dim3((m.dims[0] + 63) / 64, (B + 63) / 64, N), 256, 0, s>>>(
         B, m.dims[0], h->feat, (long long)h->S * m.dims[0], m.dims[0], batch_idx, B, h->S, st->A[0], (long long)B * m.dims[0],
-        nullptr, 0, h->d_status);
+        h->d_status);
     DBW_LAUNCHED();
     gather_labels_kernel<<<N, 128, 0, s>>>(B, h->S, h->labels, batch_idx, st->ylab);
     DBW_LAUNCHED();
@@ -834,14 +802,13 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         DBW_LAUNCHED();
     }
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
-    bf16* dzPT = nullptr;  // the dW GEMMs read dZ itself as an MN-major operand
     const int parts = B >= 64 ? 4 : 1;
     if (C <= 16)
         head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
-            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP, dzPT);
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
     else
         head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N, parts), 64, (size_t)B * 32 * 4, s>>>(
-            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP, dzPT);
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
     DBW_LAUNCHED();
     head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
                                                                               m.w_off[L - 1], m.b_off[L - 1]);
