@@ -127,7 +127,7 @@ class Job:
         if w.backups == "dtur" and self.k > 0:
             self.h.update_backups(self.d_t[r], self.b_dyn)
             b = self.b_dyn
-        self.h.round(self.X, self.d_t[r], b, w.lr, self.X, self.kept,
+        self.h.round(self.X, self.d_t[r], b, wl.learning_rate(w, self.k % self.n_rounds), self.X, self.kept,
                      batch_idx=None if self.d_idx is None else self.d_idx[r], G_ext=self.G,
                      T_worker=self.Tw, T_round=self.Tr, loss=self.loss)
         self.k += 1
@@ -136,7 +136,7 @@ class Job:
         """One round with the per-round inputs in pinned host memory and the results read back."""
         w, r = self.w, self.k % self.n_rounds
         dyn = w.backups == "dtur" and self.k > 0
-        self.h.round_host(self.X, self.h_t[r], None if dyn else self.h_b[r], w.lr, self.X,
+        self.h.round_host(self.X, self.h_t[r], None if dyn else self.h_b[r], wl.learning_rate(w, self.k % self.n_rounds), self.X,
                           h_batch_idx=None if self.h_idx is None else self.h_idx[r], G_ext=self.G,
                           h_kept=self.hk, h_T_worker=self.hTw, h_T_round=self.hTr,
                           h_loss=None if self.h_idx is None else self.hloss, h_b_out=self.hb_out if dyn else None)

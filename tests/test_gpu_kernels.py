@@ -239,6 +239,7 @@ def test_grad_fp32_matches_oracle(dims, batch, n):
                                            ([3072, 512, 256, 10], 128, 2),     # config 2's model
                                            ([72, 200, 136, 10], 40, 3),        # ragged M, N and K tails
                                            ([320, 264, 24], 264, 2),           # two layers, three row tiles
+                                           ([256, 256, 256, 10], 1024, 2),     # the paper's 2NN, batch 1024: 16 K-blocks in dW
                                            ([64, 10], 16, 3)])                 # softmax regression: no tensor-core layer
 def test_grad_bf16_tensor_cores_match_oracle(dims, batch, n):
     """BF16 operands, fp32 accumulate: the gradient agrees with the double-precision oracle on the

@@ -14,6 +14,7 @@ from .configs import (  # noqa: F401
     fixed_backups,
     init_params,
     layer_dims,
+    learning_rate,
     logical_dim,
     make_workload,
     random_regular,

@@ -172,6 +172,7 @@ class Workload:
     means_seed: int = 0
     batch: int = 0
     lr: float = 0.05
+    lr_decay: float = 1.0            # eta(k) = lr * lr_decay^k (k = 0 for the first round)
     rounds: int = 0
     backups: str = "fixed"           # "fixed" | "dtur" | "uniform"
     fixed_b: int = 0
@@ -179,7 +180,7 @@ class Workload:
     weight_rule: str = "metropolis"  # "metropolis" | "uniform"
     times: str = "shifted_exp"       # "shifted_exp" | "lognormal"
     shift: float = 1.0
-    rate_mode: str = "one"           # "one" | "uniform_0.5_2" | "stragglers"
+    rate_mode: str = "one"           # "one" | "uniform_0.5_2" | "stragglers" | "round_straggler"
     times_seed: int = 0
     init: str = "he"                 # "he" | "small" | "gaussian"
     init_seed: int = 0
@@ -209,6 +210,13 @@ CONFIGS = {
     3: dict(name="c3_reg8_n128_mlp1024_bf16", N=128, graph="regular", degree=8,
             layers=[3072, 1024, 1024, 10], precision="bf16", samples=5000, noise=0.3, batch=256,
             rounds=50, backups="dtur", times="lognormal"),
+    # Paper-shaped workloads (Section 5 and Appendix B): 6 workers with logistic regression, 10 workers
+    # with the 256-256-10 network, batch 1024, learning rate eta_0 * 0.95^k, at least one straggler per
+    # iteration.  The 256-dimensional Gaussian-mixture features stand in for the PCA-reduced images.
+    5: dict(name="p0_lrm_6workers", N=6, graph="er", er_p=0.5, layers=[256, 10], samples=4096, noise=0.5,
+            batch=1024, lr=0.2, lr_decay=0.95, rounds=60, backups="dtur", rate_mode="round_straggler", init="small"),
+    6: dict(name="p1_2nn_10workers", N=10, graph="er", er_p=0.4, layers=[256, 256, 256, 10], samples=6000, noise=0.5,
+            batch=1024, lr=1.0, lr_decay=0.95, rounds=60, backups="dtur", rate_mode="round_straggler"),
     4: dict(name="c4_reg32_n1024_mix", N=1024, graph="regular", degree=32, layers=None,
             d=1 << 20, rounds=10, backups="uniform", max_b=8, weight_rule="uniform",
             init="gaussian", init_seed=4),
@@ -314,7 +322,7 @@ def external_gradient_seed(w: Workload) -> int:
 def worker_rates(w: Workload) -> np.ndarray:
     """Per-worker exponential rate of the compute-time distribution."""
     rng = _rng(_seed(w.index, "rates"))
-    if w.rate_mode == "one":
+    if w.rate_mode in ("one", "round_straggler"):
         return np.ones(w.N)
     if w.rate_mode == "uniform_0.5_2":
         return rng.uniform(0.5, 2.0, size=w.N)
@@ -332,10 +340,19 @@ def arrival_times(w: Workload, rounds: Optional[int] = None) -> np.ndarray:
     rng = _rng(w.times_seed)
     if w.times == "shifted_exp":
         rates = worker_rates(w)
-        return w.shift + rng.exponential(1.0, size=(rounds, w.N)) / rates[None, :]
+        t = w.shift + rng.exponential(1.0, size=(rounds, w.N)) / rates[None, :]
+        if w.rate_mode == "round_straggler":     # every round one random worker takes five times as long
+            slow = rng.integers(0, w.N, size=rounds)
+            t[np.arange(rounds), slow] *= 5.0
+        return t
     if w.times == "lognormal":
         return rng.lognormal(0.0, 1.0, size=(rounds, w.N))
     raise ValueError(w.times)
+
+
+def learning_rate(w: Workload, k: int) -> float:
+    """eta(k) of round k (0-based)."""
+    return float(w.lr * w.lr_decay ** k)
 
 
 def fixed_backups(w: Workload) -> np.ndarray:
