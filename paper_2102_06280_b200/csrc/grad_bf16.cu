@@ -674,15 +674,27 @@ bool balloc(BF16State* st, T** p, size_t n) {
 // Tile width for an output with N columns: 256 halves the operand re-reads out of L2 per output byte.
 int tile_bn(int N) { return N >= 256 ? 256 : 128; }
 
-int g_tc_sm_count = 0;
+// multiprocessor count and shared-memory opt-in are per device: looked up for the current device
+int current_device_sms(int* dev_out) {
+    static int sms[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!sms[dev]) cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+    *dev_out = dev;
+    return sms[dev];
+}
 
 template <bool AMN, bool BMN>
 int run_tc_major(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
     const int bn = tile_bn(g.N);
     const int tiles_n = (g.N + bn - 1) / bn, tiles_m = (g.M + BM - 1) / BM;
     const int n_tiles = tiles_n * tiles_m * workers;
-    const int grid = n_tiles < g_tc_sm_count ? n_tiles : g_tc_sm_count;
-    static bool configured = false;
+    int dev = 0;
+    const int sms = current_device_sms(&dev);
+    if (sms <= 0) return DBW_ERR_CUDA;
+    const int grid = n_tiles < sms ? n_tiles : sms;
+    static bool configured_dev[64] = {};
+    bool& configured = configured_dev[dev];
     if (!configured) {
         DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<4, 128, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(4, 128)));
         DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 256, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 256)));
@@ -744,7 +756,6 @@ int grad_bf16_alloc(dbw_handle* h) {
         }
     }
     if (!ok) return DBW_ERR_CUDA;
-    g_tc_sm_count = h->sm_count;
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
