@@ -281,8 +281,8 @@ def run_reference(args):
     if rank != 0:
         return
     w = wl.make_workload(args.config)
-    # the whole run (warm-up included) is bounded to about two minutes of CPU work
-    budget = min(args.ref_budget, 120.0 / (args.steps + args.warmup))
+    # the whole run (warm-up included) is bounded to a minute or two of CPU work
+    budget = min(args.ref_budget, 60.0 / (args.steps + args.warmup))
     for _ in range(args.warmup):
         oracle_sample_seconds(w, 0, budget_s=budget)
     est = []
