@@ -407,7 +407,7 @@ def measure(config, local, args, dist, overrides):
     for _ in range(min(args.warmup, 3)):
         job.step_host()
     ms_e2e = timed_loop(job, args.steps, job.step_host, dist)
-    out = dict(w=job.w, ld=job.ld, ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
+    out = dict(w=job.w, ld=job.ld, mix_kernel=job.h.mix_kernel(), ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
                stage_ms={k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
                bytes=job.host_bytes_per_step(), mix_bytes=job.mix_bytes_per_launch())
     job.close()
@@ -430,7 +430,6 @@ def summary(res, world, args):
     peaks, peak_kind = measured_peaks()
     mix_ms = res["stage_ms"]["mix"]
     achieved = res["mix_bytes"] / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
-    staged = w.weight_rule == "uniform" and 64 <= w.N <= 1024 and w.N * 128 > 113 * 1024
     h2d, d2h = res["bytes"]
     out = {"value": aggregate_value(w.N, args.steps, res["ms"], world), "ms_per_step": res["ms"] / args.steps,
            "dtype": "f32" if w.precision == "fp32" else "bf16",
@@ -444,7 +443,7 @@ def summary(res, world, args):
            "e2e": {"value": aggregate_value(w.N, args.steps, res["ms_e2e"], world), "unit": UNIT,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": res["ms_e2e"] / args.steps},
            "gpu_launches": int(res["launches"]),
-           "roofline": {"kernel": "mix_staged_kernel" if staged else "mix_panel_kernel", "bound": "hbm",
+           "roofline": {"kernel": res["mix_kernel"], "bound": "hbm",
                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                         "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
                         "bytes_per_launch": res["mix_bytes"], "ms_per_launch": mix_ms},

@@ -169,6 +169,9 @@ int dbw_mix_in_place_ok(const dbw_handle* h);
  * 1 = the tensor-memory staged kernel wherever it applies (uniform weights, 64 <= N <= 1024),
  * -1 = always the direct (L2 re-read, out-of-place only) kernel. */
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols);
+/* Which mix kernel the current settings select: 0 = direct (L2 re-read), 1 = shared-memory panel,
+ * 2 = tensor-memory staged.  Negative on error. */
+int dbw_mix_kernel(const dbw_handle* h);
 
 /*
  * Algorithm 1, one iteration: gradients (dbw_grad, or G_ext when batch_idx is NULL), selection

@@ -53,6 +53,7 @@ _SIGNATURES = {
     "dbw_mix": (C.c_int, [_P, _P, _P, _P, _P, C.c_float, _P, _P, _P]),
     "dbw_mix_in_place_ok": (C.c_int, [_P]),
     "dbw_set_mix_panel": (C.c_int, [_P, C.c_int32]),
+    "dbw_mix_kernel": (C.c_int, [_P]),
     "dbw_set_param_tracking": (C.c_int, [_P, C.c_int]),
     "dbw_round": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_round_host": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P]),
@@ -205,6 +206,9 @@ class Dbw:
 
     def set_param_tracking(self, enable: bool):
         _check(lib().dbw_set_param_tracking(self._h, int(bool(enable))), "dbw_set_param_tracking")
+
+    def mix_kernel(self) -> str:
+        return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]
 
     def set_mix_panel(self, cols: int):
         _check(lib().dbw_set_mix_panel(self._h, int(cols)), "dbw_set_mix_panel")

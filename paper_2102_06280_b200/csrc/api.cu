@@ -305,6 +305,8 @@ int dbw_set_param_tracking(dbw_handle* h, int enable) {
 
 int dbw_mix_in_place_ok(const dbw_handle* h) { return h && mix_panel_fits(h) ? 1 : 0; }
 
+int dbw_mix_kernel(const dbw_handle* h) { return h ? mix_kernel_kind(h) : DBW_ERR_NULL; }
+
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols) {
     if (!h) return DBW_ERR_NULL;
     if (!(cols == 0 || cols == -1 || cols == 1 || cols == 16 || cols == 32 || cols == 64 || cols == 128)) return DBW_ERR_BAD_SHAPE;

@@ -128,6 +128,7 @@ __device__ __forceinline__ uint2 pack_bf16x4_rn(float a, float b, float c, float
     return make_uint2(lo, hi);
 }
 bool mix_panel_fits(const dbw_handle* h);
+int mix_kernel_kind(const dbw_handle* h);
 
 // mix_staged.cu
 bool mix_staged_usable(const dbw_handle* h);

@@ -160,6 +160,7 @@ static bool use_staged(const dbw_handle* h) {
 }
 
 bool mix_panel_fits(const dbw_handle* h) { return use_staged(h) || auto_group_size(h) != 0; }
+int mix_kernel_kind(const dbw_handle* h) { return use_staged(h) ? 2 : (auto_group_size(h) != 0 ? 1 : 0); }
 
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s) {
