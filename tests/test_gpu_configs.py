@@ -281,3 +281,56 @@ def test_round_host_matches_device_round():
     assert torch.equal(h_kept, sim.kept.cpu()) and torch.equal(h_Tw, sim.Tw.cpu()) and torch.equal(h_Tr, sim.Tr.cpu())
     assert torch.equal(h_loss, sim.loss.cpu())
     sim.h.close()
+
+
+@pytest.mark.parametrize("cfg,flag", [(0, 0), (2, 4)])
+def test_round_replays_from_a_cuda_graph(cfg, flag):
+    """After a warm-up call (which does the one-time allocations and kernel attributes) a round and
+    the threshold rule can be captured into a CUDA graph; replays with new inputs in the same buffers
+    give the same bits as eager calls."""
+    w = wl.make_workload(cfg) if cfg == 0 else wl.make_workload(cfg, N=16, er_p=0.35, samples=300)
+    sim = Sim(w, flag)
+    m = sim.m
+    times = wl.arrival_times(w, 4)
+    X_eager = dev(m.pack(sim.X0))
+    X_graph = X_eager.clone()
+    t_buf = dev(times[0])
+    idx_buf = dev(wl.batch_indices(w, 0))
+    dynamic = w.backups == "dtur"
+    sim.b_d.copy_(dev(wl.fixed_backups(w)) if not dynamic else torch.zeros_like(sim.b_d))
+
+    def one_round(X):
+        if dynamic:
+            sim.h.update_backups(t_buf, sim.b_d)
+        sim.h.round(X, t_buf, sim.b_d, w.lr, X, sim.kept, batch_idx=idx_buf, T_round=sim.Tr, loss=sim.loss)
+
+    # eager reference: warm-up round included
+    for k in range(4):
+        t_buf.copy_(dev(times[k])); idx_buf.copy_(dev(wl.batch_indices(w, k)))
+        one_round(X_eager)
+    torch.cuda.synchronize()
+    tr_eager = float(sim.Tr.cpu()[0])
+    # the same four rounds, rounds 1..3 replayed from a graph captured after round 0
+    sim.h.reset_backups()
+    sim.b_d.copy_(dev(wl.fixed_backups(w)) if not dynamic else torch.zeros_like(sim.b_d))
+    t_buf.copy_(dev(times[0])); idx_buf.copy_(dev(wl.batch_indices(w, 0)))
+    one_round(X_graph)                                   # warm-up / round 0, eager
+    torch.cuda.synchronize()
+    saved = X_graph.clone()
+    state = sim.h.state_export() if dynamic else None
+    b_saved = sim.b_d.clone()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one_round(X_graph)                               # capture only: nothing runs
+    X_graph.copy_(saved)
+    sim.b_d.copy_(b_saved)
+    if dynamic:
+        sim.h.state_import(state)
+    for k in range(1, 4):
+        t_buf.copy_(dev(times[k])); idx_buf.copy_(dev(wl.batch_indices(w, k)))
+        g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(X_graph, X_eager)
+    assert float(sim.Tr.cpu()[0]) == tr_eager
+    assert sim.h.status() == 0
+    sim.h.close()
