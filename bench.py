@@ -132,6 +132,27 @@ class Job:
                      T_worker=self.Tw, T_round=self.Tr, loss=self.loss)
         self.k += 1
 
+    def capture(self, rounds_per_graph: int):
+        """Capture `rounds_per_graph` consecutive rounds into one CUDA graph (launch-bound workloads).
+
+        The graph bakes in the inputs of the rounds it was captured on, so replays cycle through
+        those rounds' arrival times and batches; parameters and the threshold rule's state keep
+        evolving.  Call after the warm-up rounds (one-time allocations happen there)."""
+        torch = self.torch
+        torch.cuda.synchronize()
+        k0 = self.k
+        self._graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self._graph):
+            for _ in range(rounds_per_graph):
+                self.step()
+        self.k = k0
+        self._graph_rounds = rounds_per_graph
+
+    def step_graph(self):
+        """`rounds_per_graph` rounds by one graph launch."""
+        self._graph.replay()
+        self.k += self._graph_rounds
+
     def step_host(self):
         """One round with the per-round inputs in pinned host memory and the results read back."""
         w, r = self.w, self.k % self.n_rounds
@@ -403,11 +424,17 @@ def measure(config, local, args, dist, overrides):
     launches = binding.launch_count() - launches0
     stage_ms, stage_rounds = job.h.profile_read()
     job.h.profile(False)
+    graph_ms = None
+    if args.graph and args.steps % args.graph == 0:
+        # the same loop replayed from a CUDA graph of args.graph rounds (no stage events inside)
+        job.capture(args.graph)
+        job.step_graph()
+        graph_ms = timed_loop(job, args.steps // args.graph, job.step_graph, dist)
     # end to end: per-round inputs from pinned host memory, results read back every round
     for _ in range(min(args.warmup, 3)):
         job.step_host()
     ms_e2e = timed_loop(job, args.steps, job.step_host, dist)
-    out = dict(w=job.w, ld=job.ld, mix_kernel=job.h.mix_kernel(), ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
+    out = dict(w=job.w, ld=job.ld, mix_kernel=job.h.mix_kernel(), graph_ms=graph_ms, ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
                stage_ms={k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
                bytes=job.host_bytes_per_step(), mix_bytes=job.mix_bytes_per_launch())
     job.close()
@@ -448,6 +475,10 @@ def summary(res, world, args):
                         "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
                         "bytes_per_launch": res["mix_bytes"], "ms_per_launch": mix_ms},
            "device_status": res["status"]}
+    if res.get("graph_ms"):
+        out["cuda_graph"] = {"rounds_per_graph": args.graph, "ms_per_step": res["graph_ms"] / args.steps,
+                             "value": aggregate_value(w.N, args.steps, res["graph_ms"], world),
+                             "note": "same rounds replayed from one CUDA graph per %d rounds" % args.graph}
     flops = model_flops_per_round(w)
     if flops and res["stage_ms"]["grad"] > 0:
         out["gradients"] = {"dense_flop_per_round": flops,
@@ -467,6 +498,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--also", type=int, nargs="*", default=[3], choices=sorted(wl.CONFIGS),
                     help="further workloads summarised under other_workloads (single GPU only)")
+    ap.add_argument("--graph", type=int, default=0,
+                    help="also time the loop replayed from CUDA graphs of this many rounds (must divide --steps)")
     ap.add_argument("--samples", type=int, default=0, help="profiling aid: samples per worker instead of the config's")
     ap.add_argument("--width", type=int, default=0, help="profiling aid: columns d of the mix-only config instead of 2^20")
     args = ap.parse_args()
