@@ -15,6 +15,10 @@
  *     or retained past the call unless stated); pointers marked HOST are host memory.
  *   - all device work is enqueued on the `stream` argument (a cudaStream_t passed as void*)
  *     and is asynchronous; the caller synchronises.
+ *   - dbw_round, dbw_grad, dbw_mix, dbw_select and dbw_update_backups allocate nothing after their
+ *     first call on a handle (dbw_round's gradient workspace and a few kernel attributes are set up
+ *     then), so later calls may be captured into a CUDA graph; what a call decides on the host
+ *     (which kernel, whether a tracked bf16 copy is reused) is decided at capture time.
  *   - conditions that only the device can see (b_i outside [0, deg_i], NaN arrival time,
  *     a pipeline wait that ran out) set bits in a status word read by dbw_status(); the
  *     kernels clamp and continue, they never trap.
