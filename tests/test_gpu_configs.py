@@ -334,3 +334,22 @@ def test_round_replays_from_a_cuda_graph(cfg, flag):
     assert float(sim.Tr.cpu()[0]) == tr_eager
     assert sim.h.status() == 0
     sim.h.close()
+
+
+@pytest.mark.parametrize("cfg,flag", [(1, 0), (2, 4)])
+def test_rounds_are_reproducible_bit_for_bit(cfg, flag):
+    """No atomics on floating-point data and fixed summation orders: the same round run twice (fresh
+    handles) gives identical parameters, losses, masks and times."""
+    w = wl.make_workload(cfg, samples=400) if cfg == 1 else wl.make_workload(cfg, N=16, er_p=0.35, samples=300)
+    times = wl.arrival_times(w, 3)
+    results = []
+    for rep in range(2):
+        sim = Sim(w, flag)
+        X = dev(sim.m.pack(sim.X0))
+        for k in range(3):
+            sim.backups(k, times[k])
+            sim.gpu_round(X, times[k], wl.batch_indices(w, k), X)
+        results.append((X.clone(), sim.loss.clone(), sim.kept.clone(), sim.Tw.clone()))
+        sim.h.close()
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
