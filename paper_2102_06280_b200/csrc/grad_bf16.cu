@@ -672,7 +672,13 @@ bool balloc(BF16State* st, T** p, size_t n) {
 }
 
 // Tile width for an output with N columns: 256 halves the operand re-reads out of L2 per output byte.
-int tile_bn(int N) { return N >= 256 ? 256 : 128; }
+// The wide tile only when it still leaves at least one tile per SM (148 on B200; small problems keep
+// more CTAs busy with 128-wide tiles).
+int tile_bn(int N, int M, int workers) {
+    if (N < 256) return 128;
+    const long long wide_tiles = (long long)((N + 255) / 256) * ((M + BM - 1) / BM) * workers;
+    return wide_tiles >= 148 ? 256 : 128;
+}
 
 // multiprocessor count and shared-memory opt-in are per device: looked up for the current device
 int current_device_sms(int* dev_out) {
@@ -686,7 +692,7 @@ int current_device_sms(int* dev_out) {
 
 template <bool AMN, bool BMN>
 int run_tc_major(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
-    const int bn = tile_bn(g.N);
+    const int bn = tile_bn(g.N, g.M, workers);
     const int tiles_n = (g.N + bn - 1) / bn, tiles_m = (g.M + BM - 1) / BM;
     const int n_tiles = tiles_n * tiles_m * workers;
     int dev = 0;
@@ -747,7 +753,7 @@ int grad_bf16_alloc(dbw_handle* h) {
     if (!ok) return DBW_ERR_CUDA;
     for (int l = 0; l <= L - 2; ++l) {
         ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
-        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1]));
+        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1], B, N));
         ok = ok && make_operand_map_mn(&st->dwA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
         ok = ok && make_operand_map_mn(&st->dwB[l], st->A[l], m.dims[l], B, N);
         if (l >= 1) {
