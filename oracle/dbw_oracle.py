@@ -31,12 +31,13 @@ MIX_THEN_CORRECT = "mix_then_correct"  # Eq. 3 restricted to the kept set
 # Section 2.2: worker j waits for the first p_j(k) updates of its neighbours
 # ---------------------------------------------------------------------------
 
-def select_fastest(rowptr, col, t, b):
+def select_fastest(rowptr, col, t, b, t_edge=None):
     """Kept-neighbour mask, aligned with `col` (1 = waited for, 0 = backup).
 
     Section 2.2: worker i keeps the first p_i = deg_i - b_i updates to arrive.
     The update of neighbour j arrives at t_j; equal times are ordered by the
-    lower worker index.
+    lower worker index.  With `t_edge` (aligned with `col`) the update of
+    col[e] arrives at worker i at t_edge[e] instead (per-link delays).
     """
     n = len(rowptr) - 1
     kept = np.zeros(len(col), dtype=np.uint8)
@@ -46,7 +47,8 @@ def select_fastest(rowptr, col, t, b):
         p = deg - int(b[i])
         if p < 0 or p > deg:
             raise ValueError("b out of range for worker %d" % i)
-        order = sorted(range(lo, hi), key=lambda e: (float(t[col[e]]), int(col[e])))
+        arrive = (lambda e: float(t_edge[e])) if t_edge is not None else (lambda e: float(t[col[e]]))
+        order = sorted(range(lo, hi), key=lambda e: (arrive(e), int(col[e])))
         for e in order[:p]:
             kept[e] = 1
     return kept
@@ -57,14 +59,16 @@ def select_fastest(rowptr, col, t, b):
 # T(k) = max{T_j : j in V'}
 # ---------------------------------------------------------------------------
 
-def round_times(rowptr, col, t, b, kept):
+def round_times(rowptr, col, t, b, kept, t_edge=None):
     """(T_nbr, T_worker, T_round) of one round.
 
-    T_nbr[i]    = max of t over the kept neighbours of i (0.0 when p_i = 0);
+    T_nbr[i]    = max arrival time over the kept neighbours of i (0.0 when p_i = 0);
     a worker participates when it waits for someone or someone waits for it;
     T_worker[i] = max(t_i, T_nbr[i]) when p_i >= 1, t_i when it only participates
                   through others, 0.0 when it does not participate;
-    T_round     = max of t over the participating workers (0.0 if none).
+    T_round     = max of T_worker over the participating workers (0.0 if none).
+    Without per-link delays this is the max of t over the participating workers,
+    because every kept neighbour participates itself.
     """
     n = len(rowptr) - 1
     t = np.asarray(t, dtype=np.float64)
@@ -76,7 +80,7 @@ def round_times(rowptr, col, t, b, kept):
             if kept[e]:
                 j = int(col[e])
                 waited_for[j] = True
-                T_nbr[i] = max(T_nbr[i], t[j])
+                T_nbr[i] = max(T_nbr[i], t[j] if t_edge is None else t_edge[e])
     T_worker = np.zeros(n)
     T_round = 0.0
     for i in range(n):
@@ -86,7 +90,7 @@ def round_times(rowptr, col, t, b, kept):
         elif participating:
             T_worker[i] = t[i]
         if participating:
-            T_round = max(T_round, t[i])
+            T_round = max(T_round, T_worker[i])
     return T_nbr, T_worker, T_round
 
 

@@ -383,3 +383,41 @@ def test_loss_decreases_on_synthetic_task():
         X = r["X"]
         losses.append(r["loss"].mean())
     assert losses[-1] < 0.8 * losses[0]
+
+
+# ----------------------------------------------------------------------------- per-link arrival times
+
+def test_per_link_times_brute_force_and_reduction():
+    """With per-link delays the kept set is the p smallest (arrival, index) keys of the worker's own
+    links (brute force over subsets); link times equal to the senders' times reproduce the per-worker
+    model exactly; T_nbr is the p-th order statistic of the link times; T(k) = max T_j (Section 3.2.2)."""
+    rng = np.random.default_rng(21)
+    for rowptr, col in _small_graphs() + [wl.random_regular(16, 4, 5)]:
+        n = len(rowptr) - 1
+        deg = np.diff(rowptr)
+        for trial in range(6):
+            t = 1.0 + rng.random(n)
+            te = np.round(4 * (t[col] + rng.random(len(col)))) / 4          # delays, with ties
+            b = rng.integers(0, deg + 1)
+            kept = orc.select_fastest(rowptr, col, t, b, t_edge=te)
+            T_nbr, T_worker, T_round = orc.round_times(rowptr, col, t, b, kept, t_edge=te)
+            waited = np.zeros(n, dtype=bool)
+            waited[col[kept == 1]] = True
+            for i in range(n):
+                es = list(range(rowptr[i], rowptr[i + 1]))
+                p = int(deg[i] - b[i])
+                best = min(itertools.combinations(es, p), key=lambda s: sorted((te[e], col[e]) for e in s))
+                assert sorted(best) == [e for e in es if kept[e]]
+                ts = sorted(te[es])
+                assert T_nbr[i] == (ts[p - 1] if p >= 1 else 0.0)
+                assert T_worker[i] == (max(t[i], T_nbr[i]) if p >= 1 else (t[i] if waited[i] else 0.0))
+            part = (deg - b >= 1) | waited
+            assert T_round == (T_worker[part].max() if part.any() else 0.0)
+            # no extra delay: identical to the per-worker model
+            k0 = orc.select_fastest(rowptr, col, t, b)
+            assert np.array_equal(k0, orc.select_fastest(rowptr, col, t, b, t_edge=t[col]))
+            a0 = orc.round_times(rowptr, col, t, b, k0)
+            a1 = orc.round_times(rowptr, col, t, b, k0, t_edge=t[col])
+            assert np.array_equal(a0[0], a1[0]) and np.array_equal(a0[1], a1[1]) and a0[2] == a1[2]
+            assert a0[2] == (t[(deg - b >= 1) | np.isin(np.arange(n), col[k0 == 1])].max()
+                             if ((deg - b >= 1).any() or k0.any()) else 0.0)
