@@ -106,12 +106,24 @@ int dbw_set_dataset(dbw_handle* h, const float* feat, const int32_t* labels, int
  *             T_nbr[N]    max t over the kept neighbours (0.0 when p_i = 0);
  *             T_worker[N] max(t_i, T_nbr[i]) when p_i >= 1; t_i when i is only waited for by
  *                         others; 0.0 when i takes no part;
- *             T_round[1]  max t over the workers that take part (0.0 if none).
+ *             T_round[1]  max of T_worker over the workers that take part (0.0 if none); without
+ *                         per-link times this is the max of t over them.
  * Only comparisons are applied to t, so the outputs are bit-exact.  Any out pointer but kept
  * may be NULL.
  */
 int dbw_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kept, double* T_worker,
                double* T_nbr, double* T_round, void* stream);
+
+/*
+ * Per-link arrival times (a generalisation the paper leaves open: it takes the communication delay
+ * as negligible, Section 4).  DEVICE t_edge[nnz], aligned with col: the update of worker col[e]
+ * reaches worker i (the row of e) at t_edge[e].  While set, dbw_select / dbw_round / dbw_round_host
+ * rank worker i's neighbours by these times (ties to the lower index), T_nbr is the latest kept
+ * link time, T_worker[i] = max(t_i, T_nbr[i]) and T_round = max of T_worker over the workers that
+ * take part.  The pointer is retained, not copied; pass NULL to return to per-worker times.  The
+ * threshold rule (dbw_update_backups) keeps using the per-worker times.
+ */
+int dbw_set_edge_times(dbw_handle* h, const double* t_edge);
 
 /*
  * dbw_select for callers that must not allocate.  (The paper has no counterpart: this is an

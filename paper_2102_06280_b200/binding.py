@@ -47,6 +47,7 @@ _SIGNATURES = {
     "dbw_init": (C.c_int, [C.POINTER(_P), C.c_int32, C.c_int64, C.c_int64, _P, _P, C.POINTER(_ModelDesc), C.c_uint32, C.c_int]),
     "dbw_destroy": (C.c_int, [_P]),
     "dbw_set_dataset": (C.c_int, [_P, _P, _P, C.c_int32]),
+    "dbw_set_edge_times": (C.c_int, [_P, _P]),
     "dbw_select": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_select_static": (C.c_int, [C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_grad": (C.c_int, [_P, _P, _P, _P, _P, _P]),
@@ -189,6 +190,10 @@ class Dbw:
     def set_dataset(self, feat, labels, S: int):
         self._keep = (feat, labels)
         _check(lib().dbw_set_dataset(self._h, _ptr(feat), _ptr(labels), int(S)), "dbw_set_dataset")
+
+    def set_edge_times(self, t_edge):
+        self._keep_edge = t_edge
+        _check(lib().dbw_set_edge_times(self._h, _ptr(t_edge)), "dbw_set_edge_times")
 
     def select(self, t, b, kept, T_worker=None, T_nbr=None, T_round=None):
         _check(lib().dbw_select(self._h, _ptr(t), _ptr(b), _ptr(kept), _ptr(T_worker), _ptr(T_nbr), _ptr(T_round),

@@ -257,6 +257,12 @@ int dbw_set_dataset(dbw_handle* h, const float* feat, const int32_t* labels, int
     return DBW_OK;
 }
 
+int dbw_set_edge_times(dbw_handle* h, const double* t_edge) {
+    if (!h) return DBW_ERR_NULL;
+    h->t_edge = t_edge;
+    return DBW_OK;
+}
+
 int dbw_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kept, double* T_worker, double* T_nbr,
                double* T_round, void* stream) {
     if (!h || !t || !b || !kept) return DBW_ERR_NULL;

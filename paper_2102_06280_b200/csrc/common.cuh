@@ -73,6 +73,8 @@ struct dbw_handle {
     uint32_t* d_ticket = nullptr;    // [1] block ticket of the selection kernel (kept zero between calls)
     double* d_Tnbr_ws = nullptr;     // [N]
 
+    const double* t_edge = nullptr;  // optional per-link arrival times (caller-owned, DEVICE, aligned with col)
+
     dbw::MixPlan plan;
     int mix_panel_cols = 0;  // 0 = automatic
 

@@ -73,7 +73,8 @@ __device__ __forceinline__ float edge_weight(bool uniform, int p_i, int p_j) {
 // per-worker and per-round times, which need to know who is waited for by whom.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-              const double* __restrict__ t, const int32_t* __restrict__ b, uint8_t* __restrict__ kept,
+              const double* __restrict__ t, const double* __restrict__ t_edge, const int32_t* __restrict__ b,
+              uint8_t* __restrict__ kept,
               double* __restrict__ T_nbr_ws, double* T_nbr_out, double* T_worker, double* T_round,
               uint32_t* waited, uint32_t* ticket, uint32_t* status, MixPlan plan, int build_plan,
               int uniform) {
@@ -89,12 +90,13 @@ select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restri
             const int e = lo + base + lane;
             const bool valid = e < hi;
             const int j = valid ? col[e] : 0x7fffffff;
-            const double tj = valid ? order_time(t[j], status) : 0.0;
+            // arrival of col[e]'s update at worker i: the sender's time, or the link's own time
+            const double tj = valid ? order_time(t_edge ? t_edge[e] : t[j], status) : 0.0;
             int rank = 0;
             for (int base2 = 0; base2 < deg; base2 += 32) {
                 const int e2 = lo + base2 + lane;
                 const int j2 = e2 < hi ? col[e2] : 0x7fffffff;
-                const double t2 = e2 < hi ? order_time(t[j2], status) : 0.0;
+                const double t2 = e2 < hi ? order_time(t_edge ? t_edge[e2] : t[j2], status) : 0.0;
                 const int n2 = min(32, deg - base2);
                 for (int s = 0; s < n2; ++s) {
                     const double ts = __shfl_sync(0xffffffffu, t2, s);
@@ -145,8 +147,9 @@ select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restri
         const double tw = order_time(t[w], status);
         const double tn = __ldcg(&T_nbr_ws[w]);
         if (T_nbr_out) T_nbr_out[w] = tn;
-        if (T_worker) T_worker[w] = p >= 1 ? fmax(tw, tn) : (part ? tw : 0.0);
-        if (part) tr = fmax(tr, tw);
+        const double twk = p >= 1 ? fmax(tw, tn) : (part ? tw : 0.0);
+        if (T_worker) T_worker[w] = twk;
+        if (part) tr = fmax(tr, twk);  // T(k) = max of T_j over the participating workers
         waited[w] = 0u;
     }
     tr = warp_max(tr);
@@ -193,7 +196,7 @@ int launch_select(dbw_handle* h, const double* t, const int32_t* b, uint8_t* kep
                   double* T_nbr, double* T_round, bool build_plan, cudaStream_t s) {
     const int blocks = (h->N + kWarpsPerBlock - 1) / kWarpsPerBlock;
     select_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(
-        h->N, h->d_rowptr, h->d_col, t, b, kept, h->d_Tnbr_ws, T_nbr, T_worker, T_round, h->d_waited,
+        h->N, h->d_rowptr, h->d_col, t, h->t_edge, b, kept, h->d_Tnbr_ws, T_nbr, T_worker, T_round, h->d_waited,
         h->d_ticket, h->d_status, h->plan, build_plan ? 1 : 0, (h->flags & DBW_WEIGHT_UNIFORM) ? 1 : 0);
     DBW_LAUNCHED();
     return DBW_OK;
@@ -258,7 +261,7 @@ extern "C" int dbw_select_static(int32_t N, const int32_t* rowptr, const int32_t
     // the array keeps whatever the previous call left: ticket, status and flags must start at zero
     DBW_CUDA(cudaMemsetAsync(base, 0, dbw::kStaticFlagsOff + sizeof(uint32_t) * (size_t)N, s));
     const int blocks = (N + dbw::kWarpsPerBlock - 1) / dbw::kWarpsPerBlock;
-    dbw::select_kernel<<<blocks, dbw::kWarpsPerBlock * 32, 0, s>>>(N, rowptr, col, t, b, kept, tnbr, T_nbr, T_worker,
+    dbw::select_kernel<<<blocks, dbw::kWarpsPerBlock * 32, 0, s>>>(N, rowptr, col, t, nullptr, b, kept, tnbr, T_nbr, T_worker,
                                                                    T_round, waited, ticket, status, dbw::MixPlan{}, 0, 0);
     DBW_LAUNCHED();
     if (status_out) DBW_CUDA(cudaMemcpyAsync(status_out, status, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));

@@ -328,3 +328,38 @@ def test_degenerate_sizes():
     assert not np.any(Xd.cpu().numpy()[:, d:])
     assert np.array_equal(kept.cpu().numpy(), r["kept"])
     h.close()
+
+
+@pytest.mark.parametrize("name", ["ring8", "complete40", "reg4_32", "er64", "reg32_256"])
+def test_selection_with_per_link_times_bit_exact(name):
+    p = _dbw()
+    rowptr, col = GRAPHS[name]()
+    n, nnz = len(rowptr) - 1, len(col)
+    deg = np.diff(rowptr)
+    h = p.Dbw(rowptr, col, d=8)
+    rng = np.random.default_rng(31)
+    X = rng.standard_normal((n, 8)).astype(np.float32)
+    G = rng.standard_normal((n, 8)).astype(np.float32)
+    for trial in range(4):
+        t = 1.0 + rng.exponential(1.0, size=n)
+        te = np.round(4 * (t[col] + rng.random(nnz))) / 4                 # link delays, with ties
+        b = rng.integers(0, deg + 1)
+        h.set_edge_times(dev(te))
+        kept, Tw, Tn, Tr = _select_gpu(h, n, nnz, t, b)
+        ref = orc.select_fastest(rowptr, col, t, b, t_edge=te)
+        assert np.array_equal(kept, ref)
+        rTn, rTw, rTr = orc.round_times(rowptr, col, t, b, ref, t_edge=te)
+        assert np.array_equal(Tn, rTn) and np.array_equal(Tw, rTw) and Tr == rTr
+        # the whole round follows the link-time selection
+        out = torch.empty(n, 8, device="cuda")
+        kd = torch.zeros(nnz, dtype=torch.uint8, device="cuda")
+        h.round(dev(X), dev(t), dev(b.astype(np.int32)), 0.1, out, kd, G_ext=dev(G))
+        torch.cuda.synchronize()
+        ws, we = orc.mixing_weights(rowptr, col, b, ref)
+        assert np.array_equal(kd.cpu().numpy(), ref)
+        assert row_rel_err(out.cpu().numpy(), orc.mix_update(rowptr, col, X, G, ws, we, 0.1)) <= 1e-5
+        h.set_edge_times(None)                                            # back to per-worker times
+        kept0, *_ = _select_gpu(h, n, nnz, t, b)
+        assert np.array_equal(kept0, orc.select_fastest(rowptr, col, t, b))
+    assert h.status() == 0
+    h.close()
