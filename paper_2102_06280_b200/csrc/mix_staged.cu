@@ -162,18 +162,34 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
     };
     auto gather = [&](int pn) {  // every output row of the panel out of shared memory
         const long long c = (long long)pn * 32 + 4 * slot;
-        for (int i = grp; i < N; i += kConsWarps * 4) {
-            float4 acc = panel[(size_t)i * 8 + slot];
-            const uint4* lp = reinterpret_cast<const uint4*>(lists + (size_t)i * prow);
-            const int nb = nblk[i];
-            for (int kb = 0; kb < nb; ++kb) {
-                const uint4 u = lp[kb];
-                const float4 v0 = panel[(size_t)(u.x & 0xffffu) * 8 + slot], v1 = panel[(size_t)(u.x >> 16) * 8 + slot];
-                const float4 v2 = panel[(size_t)(u.y & 0xffffu) * 8 + slot], v3 = panel[(size_t)(u.y >> 16) * 8 + slot];
-                const float4 v4 = panel[(size_t)(u.z & 0xffffu) * 8 + slot], v5 = panel[(size_t)(u.z >> 16) * 8 + slot];
-                const float4 v6 = panel[(size_t)(u.w & 0xffffu) * 8 + slot], v7 = panel[(size_t)(u.w >> 16) * 8 + slot];
-                add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
-                add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
+        // Flattened loop over (row, list block) with the NEXT block's indices (of this row, or of the
+        // group's next row together with that row's own segment) fetched before the current block's
+        // eight rows are gathered, so that no shared-memory round trip sits between two gathers.
+        int i = grp;
+        if (i >= N) return;
+        const uint4* lp = reinterpret_cast<const uint4*>(lists + (size_t)i * prow);
+        int nb = max((int)nblk[i], 1), kb = 0;  // a row without kept neighbours gathers one all-padding block
+        uint4 u = lp[0];
+        float4 acc = panel[(size_t)i * 8 + slot];
+        while (true) {
+            const bool last = kb + 1 >= nb;
+            const int i2 = i + kConsWarps * 4;
+            const bool more = !last || i2 < N;
+            const uint4* lp2 = last ? reinterpret_cast<const uint4*>(lists + (size_t)i2 * prow) : lp;
+            uint4 un = u;
+            float4 acc2 = acc;
+            if (more) un = lp2[last ? 0 : kb + 1];
+            if (last && i2 < N) acc2 = panel[(size_t)i2 * 8 + slot];
+            const float4 v0 = panel[(size_t)(u.x & 0xffffu) * 8 + slot], v1 = panel[(size_t)(u.x >> 16) * 8 + slot];
+            const float4 v2 = panel[(size_t)(u.y & 0xffffu) * 8 + slot], v3 = panel[(size_t)(u.y >> 16) * 8 + slot];
+            const float4 v4 = panel[(size_t)(u.z & 0xffffu) * 8 + slot], v5 = panel[(size_t)(u.z >> 16) * 8 + slot];
+            const float4 v6 = panel[(size_t)(u.w & 0xffffu) * 8 + slot], v7 = panel[(size_t)(u.w >> 16) * 8 + slot];
+            add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
+            add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
+            u = un;
+            if (!last) {
+                ++kb;
+                continue;
             }
             const float w = scale[i];
             acc.x *= w; acc.y *= w; acc.z *= w; acc.w *= w;
@@ -187,6 +203,12 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
                 *reinterpret_cast<float4*>(a.Xout + (size_t)i * a.ld + c) = acc;
                 if (a.shadow) *reinterpret_cast<uint2*>(a.shadow + (size_t)i * a.ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
             }
+            if (i2 >= N) break;
+            i = i2;
+            lp = lp2;
+            nb = max((int)nblk[i], 1);
+            kb = 0;
+            acc = acc2;
         }
     };
 
