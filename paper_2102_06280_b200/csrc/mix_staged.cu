@@ -5,8 +5,9 @@
 // fill shared memory, so there is no room for a second panel buffer, and with about 30 terms per
 // output the gather out of shared memory takes longer than the HBM stream.  To overlap the two,
 // eight producer warps stream the next panel of X and G from HBM (128-bit loads, x - lr*g formed
-// in registers) and park it in the SM's tensor memory with tcgen05.st, while sixteen consumer warps
-// gather the current panel out of shared memory.  When both are done the producers move the parked
+// in registers) and park it in the SM's tensor memory with tcgen05.st, while twenty-four consumer
+// warps gather the current panel out of shared memory (the gather waits on shared-memory round
+// trips, so it wants every warp the SM can hold).  When both are done the producers move the parked
 // panel from tensor memory into shared memory (tcgen05.ld + 128-bit shared stores) and the roles
 // repeat.  The neighbour lists (16-bit indices, built once per launch from the mixing plan) stay in
 // shared memory for the whole launch.  HBM traffic is the algorithmic 12 bytes per element; a panel
@@ -17,34 +18,28 @@ namespace dbw {
 
 namespace {
 
-constexpr int kProdWarps = 8, kConsWarps = 16;
-constexpr int kThreads = (kProdWarps + kConsWarps) * 32;  // 768
+constexpr int kProdWarps = 8, kConsWarps = 24;
+constexpr int kThreads = (kProdWarps + kConsWarps) * 32;  // 1024
 constexpr int kTmemCols = 256;                            // 128 lanes x 256 columns x 4 B = one 1024 x 32 panel
 constexpr int kMaxN = 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float4 (&v)[8]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float4 (&v)[4]) {
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
         ::"r"(taddr), "f"(v[0].x), "f"(v[0].y), "f"(v[0].z), "f"(v[0].w), "f"(v[1].x), "f"(v[1].y), "f"(v[1].z), "f"(v[1].w),
-        "f"(v[2].x), "f"(v[2].y), "f"(v[2].z), "f"(v[2].w), "f"(v[3].x), "f"(v[3].y), "f"(v[3].z), "f"(v[3].w), "f"(v[4].x),
-        "f"(v[4].y), "f"(v[4].z), "f"(v[4].w), "f"(v[5].x), "f"(v[5].y), "f"(v[5].z), "f"(v[5].w), "f"(v[6].x), "f"(v[6].y),
-        "f"(v[6].z), "f"(v[6].w), "f"(v[7].x), "f"(v[7].y), "f"(v[7].z), "f"(v[7].w)
+        "f"(v[2].x), "f"(v[2].y), "f"(v[2].z), "f"(v[2].w), "f"(v[3].x), "f"(v[3].y), "f"(v[3].z), "f"(v[3].w)
         : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float4 (&v)[8]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float4 (&v)[4]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=f"(v[0].x), "=f"(v[0].y), "=f"(v[0].z), "=f"(v[0].w), "=f"(v[1].x), "=f"(v[1].y), "=f"(v[1].z), "=f"(v[1].w),
-          "=f"(v[2].x), "=f"(v[2].y), "=f"(v[2].z), "=f"(v[2].w), "=f"(v[3].x), "=f"(v[3].y), "=f"(v[3].z), "=f"(v[3].w),
-          "=f"(v[4].x), "=f"(v[4].y), "=f"(v[4].z), "=f"(v[4].w), "=f"(v[5].x), "=f"(v[5].y), "=f"(v[5].z), "=f"(v[5].w),
-          "=f"(v[6].x), "=f"(v[6].y), "=f"(v[6].z), "=f"(v[6].w), "=f"(v[7].x), "=f"(v[7].y), "=f"(v[7].z), "=f"(v[7].w)
+          "=f"(v[2].x), "=f"(v[2].y), "=f"(v[2].z), "=f"(v[2].w), "=f"(v[3].x), "=f"(v[3].y), "=f"(v[3].z), "=f"(v[3].w)
         : "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -120,23 +115,23 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
     auto stage = [&](int pn) {  // HBM -> registers -> tensor memory
         const long long c = (long long)pn * 32 + 4 * slot;
         const bool c_ok = c < a.ld;
-        for (int bt = 0; bt < n_its; bt += 8) {
-            float4 x[8], g[8];
+        for (int bt = 0; bt < n_its; bt += 4) {
+            float4 x[4], g[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 4; ++u) {
                 const int r = (bt + u) * 32 + p_row;
                 const bool ok = c_ok && r < N;
                 x[u] = ok ? ldg4(a.X + (size_t)r * a.ld + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             if (!a.mix_then_correct) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     const int r = (bt + u) * 32 + p_row;
                     const bool ok = c_ok && r < N;
                     g[u] = ok ? ldg4(a.G + (size_t)r * a.ld + c) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     const int r = (bt + u) * 32 + p_row;
                     const float nlr = -((a.lr_pw && r < N) ? a.lr_pw[r] : a.lr);
                     x[u].x = fmaf(nlr, g[u].x, x[u].x);
@@ -145,16 +140,16 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
                     x[u].w = fmaf(nlr, g[u].w, x[u].w);
                 }
             }
-            tmem_st32(p_taddr + (uint32_t)(4 * bt), x);
+            tmem_st16(p_taddr + (uint32_t)(4 * bt), x);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     };
     auto unpark = [&]() {  // tensor memory -> shared-memory panel
-        for (int bt = 0; bt < n_its; bt += 8) {
-            float4 x[8];
-            tmem_ld32(p_taddr + (uint32_t)(4 * bt), x);
+        for (int bt = 0; bt < n_its; bt += 4) {
+            float4 x[4];
+            tmem_ld16(p_taddr + (uint32_t)(4 * bt), x);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 4; ++u) {
                 const int r = (bt + u) * 32 + p_row;
                 if (r < N) panel[(size_t)r * 8 + slot] = x[u];
             }
