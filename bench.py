@@ -36,7 +36,7 @@ DEFAULT_CONFIG = 4
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix kernel, from the ncu captures
 # summarised under profiles/ (small case scaled by the columns processed); None = not captured for
 # this workload or the kernel changed since.
-MIX_TRAFFIC_BYTES = {4: (537.0e6 + 219.0e6) * 16}
+MIX_TRAFFIC_BYTES = {4: (537.1e6 + 220.4e6) * 16}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
