@@ -127,10 +127,24 @@ class Job:
         if w.backups == "dtur" and self.k > 0:
             self.h.update_backups(self.d_t[r], self.b_dyn)
             b = self.b_dyn
-        self.h.round(self.X, self.d_t[r], b, wl.learning_rate(w, self.k % self.n_rounds), self.X, self.kept,
+        out = self._out()
+        self.h.round(self.X, self.d_t[r], b, wl.learning_rate(w, self.k % self.n_rounds), out, self.kept,
                      batch_idx=None if self.d_idx is None else self.d_idx[r], G_ext=self.G,
                      T_worker=self.Tw, T_round=self.Tr, loss=self.loss)
+        self._swap(out)
         self.k += 1
+
+    def _out(self):
+        """X itself where the selected mix kernel may run in place, else a second buffer (ping-pong)."""
+        if self.h.mix_in_place_ok():
+            return self.X
+        if getattr(self, "X2", None) is None:
+            self.X2 = self.torch.empty_like(self.X)
+        return self.X2
+
+    def _swap(self, out):
+        if out is not self.X:
+            self.X, self.X2 = out, self.X
 
     def capture(self, rounds_per_graph: int):
         """Capture `rounds_per_graph` consecutive rounds into one CUDA graph (launch-bound workloads).
@@ -157,11 +171,13 @@ class Job:
         """One round with the per-round inputs in pinned host memory and the results read back."""
         w, r = self.w, self.k % self.n_rounds
         dyn = w.backups == "dtur" and self.k > 0
-        self.h.round_host(self.X, self.h_t[r], None if dyn else self.h_b[r], wl.learning_rate(w, self.k % self.n_rounds), self.X,
+        out = self._out()
+        self.h.round_host(self.X, self.h_t[r], None if dyn else self.h_b[r], wl.learning_rate(w, self.k % self.n_rounds), out,
                           h_batch_idx=None if self.h_idx is None else self.h_idx[r], G_ext=self.G,
                           h_kept=self.hk, h_T_worker=self.hTw, h_T_round=self.hTr,
                           h_loss=None if self.h_idx is None else self.hloss, h_b_out=self.hb_out if dyn else None)
         self.torch.cuda.current_stream().synchronize()      # the caller reads the round's results
+        self._swap(out)
         self.k += 1
 
     def host_bytes_per_step(self):
@@ -397,7 +413,8 @@ def run_ours(args):
     line = {"metric": METRIC, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic"}
     line.update(summary(res, world, args))
-    line["roofline"]["traffic"] = MIX_TRAFFIC_BYTES.get(args.config) if not overrides else None
+    line["roofline"]["traffic"] = (MIX_TRAFFIC_BYTES.get(args.config)
+                                   if not overrides and res["mix_kernel"] == "mix_staged_kernel" else None)
     line["clocks"] = clocks
     if extra:
         line["other_workloads"] = extra
@@ -414,6 +431,8 @@ def measure(config, local, args, dist, overrides):
     import torch
     from paper_2102_06280_b200 import binding
     job = Job(config, device=local, **overrides)
+    if args.mix_panel is not None:
+        job.h.set_mix_panel(args.mix_panel)
     for _ in range(args.warmup):
         job.step()
     torch.cuda.synchronize()
@@ -500,6 +519,8 @@ def main():
                     help="further workloads summarised under other_workloads (single GPU only)")
     ap.add_argument("--graph", type=int, default=0,
                     help="also time the loop replayed from CUDA graphs of this many rounds (must divide --steps)")
+    ap.add_argument("--mix-panel", type=int, default=None,
+                    help="expert knob passed to dbw_set_mix_panel (1 = staged kernel, 2 = tensor-core kernel, 16..128 = panel width)")
     ap.add_argument("--samples", type=int, default=0, help="profiling aid: samples per worker instead of the config's")
     ap.add_argument("--width", type=int, default=0, help="profiling aid: columns d of the mix-only config instead of 2^20")
     args = ap.parse_args()

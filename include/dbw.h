@@ -183,10 +183,13 @@ int dbw_mix_in_place_ok(const dbw_handle* h);
 /* Expert knob: columns per shared-memory panel of the mix kernel: 0 = automatic, 16 / 32 / 64 /
  * 128 = fixed (falls back to the direct kernel when N * cols * 4 bytes exceed shared memory),
  * 1 = the tensor-memory staged kernel wherever it applies (uniform weights, 64 <= N <= 1024),
+ * 2 = the tensor-core kernel wherever it applies (uniform weights, 256 <= N <= 1024): the mix as a
+ *     dense product with the 0/1 selection matrix, every fp32 value split exactly into three BF16
+ *     pieces, fp32 accumulation; with N > 512 it cannot run in place (dbw_mix_in_place_ok() = 0),
  * -1 = always the direct (L2 re-read, out-of-place only) kernel. */
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols);
 /* Which mix kernel the current settings select: 0 = direct (L2 re-read), 1 = shared-memory panel,
- * 2 = tensor-memory staged.  Negative on error. */
+ * 2 = tensor-memory staged, 3 = tensor-core.  Negative on error. */
 int dbw_mix_kernel(const dbw_handle* h);
 
 /*

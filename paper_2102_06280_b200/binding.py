@@ -213,7 +213,7 @@ class Dbw:
         _check(lib().dbw_set_param_tracking(self._h, int(bool(enable))), "dbw_set_param_tracking")
 
     def mix_kernel(self) -> str:
-        return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]
+        return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel", "mix_tc_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]
 
     def set_mix_panel(self, cols: int):
         _check(lib().dbw_set_mix_panel(self._h, int(cols)), "dbw_set_mix_panel")

@@ -114,6 +114,7 @@ void free_all(dbw_handle* h) {
     h->prof_events.clear();
     grad_fp32_free(h);
     grad_bf16_free(h);
+    mix_tc_free(h);
     void* ptrs[] = {h->d_rowptr, h->d_col, h->d_links, h->d_covered, h->d_epoch, h->d_status, h->d_waited,
                     h->d_ticket, h->d_Tnbr_ws, h->plan.idx, h->plan.w, h->plan.w_self, h->plan.cnt, h->d_G,
                     h->s_t, h->s_b, h->s_bidx, h->s_kept, h->s_Tw, h->s_Tr, h->s_loss};
@@ -315,7 +316,7 @@ int dbw_mix_kernel(const dbw_handle* h) { return h ? mix_kernel_kind(h) : DBW_ER
 
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols) {
     if (!h) return DBW_ERR_NULL;
-    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 16 || cols == 32 || cols == 64 || cols == 128)) return DBW_ERR_BAD_SHAPE;
+    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 2 || cols == 16 || cols == 32 || cols == 64 || cols == 128)) return DBW_ERR_BAD_SHAPE;
     h->mix_panel_cols = cols;
     return DBW_OK;
 }

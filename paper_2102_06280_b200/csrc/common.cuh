@@ -46,6 +46,7 @@ struct MixPlan {
 };
 
 struct BF16State;  // tensor-core gradient path (grad_bf16.cu)
+struct TcMixState;  // tensor-core mix (mix_tc.cu)
 
 }  // namespace dbw
 
@@ -77,6 +78,7 @@ struct dbw_handle {
 
     dbw::MixPlan plan;
     int mix_panel_cols = 0;  // 0 = automatic
+    dbw::TcMixState* mix_tc = nullptr;  // selection matrix and tensor map of the tensor-core mix (lazy)
 
     // model / gradient path
     bool has_model = false;
@@ -136,6 +138,13 @@ int mix_kernel_kind(const dbw_handle* h);
 bool mix_staged_usable(const dbw_handle* h);
 int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                       uint16_t* shadow, cudaStream_t s);
+
+// mix_tc.cu
+bool mix_tc_usable(const dbw_handle* h);
+bool mix_tc_in_place_ok(const dbw_handle* h);
+void mix_tc_free(dbw_handle* h);
+int launch_mix_tc(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+                  uint16_t* shadow, cudaStream_t s);
 
 // dtur.cu
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);

@@ -118,7 +118,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
 
 int auto_group_size(const dbw_handle* h) {
     if (h->mix_panel_cols < 0) return 0;  // direct kernel forced
-    if (h->mix_panel_cols == 1) return 0; // staged kernel forced (handled by the caller)
+    if (h->mix_panel_cols == 1 || h->mix_panel_cols == 2) return 0; // staged / tensor-core kernel forced (handled by the caller)
     if (h->mix_panel_cols) return ((size_t)h->N * h->mix_panel_cols * 4 <= (size_t)h->smem_optin) ? h->mix_panel_cols / 4 : 0;
     // widest panel whose staging buffer still lets two CTAs share an SM
     const size_t budget = (size_t)(h->smem_optin) / 2 - 1024;
@@ -159,8 +159,11 @@ static bool use_staged(const dbw_handle* h) {
     return h->mix_panel_cols == 0 && auto_group_size(h) < 8;
 }
 
-bool mix_panel_fits(const dbw_handle* h) { return use_staged(h) || auto_group_size(h) != 0; }
-int mix_kernel_kind(const dbw_handle* h) { return use_staged(h) ? 2 : (auto_group_size(h) != 0 ? 1 : 0); }
+// The tensor-core kernel (dense 0/1 selection product) when asked for and applicable.
+static bool use_tc(const dbw_handle* h) { return h->mix_panel_cols == 2 && mix_tc_usable(h); }
+
+bool mix_panel_fits(const dbw_handle* h) { return use_tc(h) ? mix_tc_in_place_ok(h) : (use_staged(h) || auto_group_size(h) != 0); }
+int mix_kernel_kind(const dbw_handle* h) { return use_tc(h) ? 3 : use_staged(h) ? 2 : (auto_group_size(h) != 0 ? 1 : 0); }
 
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s) {
@@ -169,6 +172,7 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
     uint16_t* shadow = (h->track_params && h->d_shadow) ? h->d_shadow : nullptr;
     h->shadow_valid = shadow != nullptr;
     h->shadow_of = X_out;
+    if (use_tc(h)) return launch_mix_tc(h, X, G, lr, lr_pw, X_out, shadow, s);
     if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, shadow, s);
     switch (auto_group_size(h)) {
         case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, shadow, s);

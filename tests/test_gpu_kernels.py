@@ -123,7 +123,7 @@ def test_mix_matches_oracle(name, d, rule, order):
     ws, we = orc.mixing_weights(rowptr, col, b, kept, rule)
     ref = orc.mix_update(rowptr, col, X, G, ws, we, 0.05, order)
     Xd, Gd, kd, bd = dev(X), dev(G), dev(kept), dev(b.astype(np.int32))
-    for panel in (0, 1, 16, 32, 64, 128, -1):
+    for panel in (0, 1, 2, 16, 32, 64, 128, -1):
         h.set_mix_panel(panel)
         out = torch.full_like(Xd, float("nan"))
         h.mix(Xd, Gd, kd, bd, 0.05, out)
@@ -144,6 +144,54 @@ def test_mix_matches_oracle(name, d, rule, order):
     torch.cuda.synchronize()
     ref = orc.mix_update(rowptr, col, X, G, ws, we, lrw.astype(np.float64), order)
     assert row_rel_err(out.cpu().numpy(), ref) <= 1e-5
+    assert h.status() == 0
+    h.close()
+
+
+@pytest.mark.parametrize("n,deg,d,order", [(320, 16, 1000, "local_then_mix"), (700, 16, 1300, "mix_then_correct"),
+                                           (1000, 32, 2052, "local_then_mix")])
+def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
+    """The dense 0/1-selection product on the tensor cores (three exact BF16 pieces per fp32 value): worker
+    counts that leave ragged row tiles and K chunks, widths that leave a ragged last panel, both update
+    orders, per-worker learning rates, in place where one CTA pair owns a panel, run-to-run reproducible."""
+    p = _dbw()
+    rowptr, col = wl.random_regular(n, deg, 21)
+    degs = np.diff(rowptr)
+    flags = p.WEIGHT_UNIFORM | (p.ORDER_MIX_THEN_CORRECT if order == "mix_then_correct" else 0)
+    h = p.Dbw(rowptr, col, d=d, ld=d, flags=flags)
+    h.set_mix_panel(2)
+    assert h.mix_kernel() == "mix_tc_kernel"
+    assert h.mix_in_place_ok() == (n <= 512)
+    rng = np.random.default_rng(12)
+    X = rng.standard_normal((n, d), dtype=np.float32) * np.float32(3.0)
+    X[:, ::7] *= np.float32(1e-4)                          # small and large magnitudes side by side
+    G = rng.standard_normal((n, d), dtype=np.float32)
+    t = 1.0 + rng.exponential(1.0, size=n)
+    b = rng.integers(0, np.minimum(degs, 8) + 1)
+    b[0] = degs[0]
+    kept = orc.select_fastest(rowptr, col, t, b)
+    ws, we = orc.mixing_weights(rowptr, col, b, kept, "uniform")
+    lrw = (0.01 + 0.1 * rng.random(n)).astype(np.float32)
+    Xd, Gd, kd, bd = dev(X), dev(G), dev(kept), dev(b.astype(np.int32))
+    for lr, lr_pw in ((0.05, None), (0.0, lrw)):
+        ref = orc.mix_update(rowptr, col, X, G, ws, we, lr if lr_pw is None else lr_pw.astype(np.float64), order)
+        out = torch.full_like(Xd, float("nan"))
+        h.mix(Xd, Gd, kd, bd, lr, out, lr_per_worker=None if lr_pw is None else dev(lr_pw))
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        assert row_rel_err(got, ref) <= 1e-5
+        again = torch.empty_like(Xd)
+        h.mix(Xd, Gd, kd, bd, lr, again, lr_per_worker=None if lr_pw is None else dev(lr_pw))
+        torch.cuda.synchronize()
+        assert np.array_equal(again.cpu().numpy(), got)
+        if h.mix_in_place_ok():
+            inpl = Xd.clone()
+            h.mix(inpl, Gd, kd, bd, lr, inpl, lr_per_worker=None if lr_pw is None else dev(lr_pw))
+            torch.cuda.synchronize()
+            assert np.array_equal(inpl.cpu().numpy(), got)
+        else:
+            with pytest.raises(p.DbwError):
+                h.mix(Xd, Gd, kd, bd, lr, Xd)
     assert h.status() == 0
     h.close()
 
