@@ -455,7 +455,8 @@ def measure(config, local, args, dist, overrides):
     ms_e2e = timed_loop(job, args.steps, job.step_host, dist)
     out = dict(w=job.w, ld=job.ld, mix_kernel=job.h.mix_kernel(), graph_ms=graph_ms, ms=ms, ms_e2e=ms_e2e, launches=launches, status=job.h.status(),
                stage_ms={k: v / max(stage_rounds, 1) for k, v in stage_ms.items()},
-               bytes=job.host_bytes_per_step(), mix_bytes=job.mix_bytes_per_launch())
+               bytes=job.host_bytes_per_step(), mix_bytes=job.mix_bytes_per_launch(),
+               kept_last=int(job.kept.sum().item()), sms=torch.cuda.get_device_properties(local).multi_processor_count)
     job.close()
     del job
     torch.cuda.empty_cache()
@@ -494,6 +495,16 @@ def summary(res, world, args):
                         "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
                         "bytes_per_launch": res["mix_bytes"], "ms_per_launch": mix_ms},
            "device_status": res["status"]}
+    # The second roofline of the mix: every output element needs (1 + kept neighbours) fp32 operands out
+    # of on-chip storage; shared memory delivers 128 bytes per clock and SM.  With ~30 terms per output
+    # (the mix-only workload) this bound, not HBM, is the binding one.
+    smem_peak = 128.0 * res["sms"] * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e9
+    operand_bytes = 4.0 * (w.N + res["kept_last"]) * res["ld"]
+    operand_rate = operand_bytes / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
+    out["roofline"]["operand_delivery"] = {
+        "terms_per_output": 1.0 + res["kept_last"] / w.N, "bytes_per_launch": operand_bytes, "achieved": operand_rate,
+        "peak": smem_peak, "unit": "GB/s", "frac": operand_rate / smem_peak,
+        "peak_kind": "128 B/clk/SM x %d SMs x %.0f MHz (shared-memory data pipe, nominal)" % (res["sms"], peaks.get("sm_max_mhz", 1965.0))}
     if res.get("graph_ms"):
         out["cuda_graph"] = {"rounds_per_graph": args.graph, "ms_per_step": res["graph_ms"] / args.steps,
                              "value": aggregate_value(w.N, args.steps, res["graph_ms"], world),
