@@ -26,8 +26,11 @@ if ROOT not in sys.path:
 
 
 def run(config: int, rounds: Optional[int] = None, dynamic: bool = True, bf16: bool = False, device: int = 0,
-        **overrides) -> Dict[str, np.ndarray]:
-    """One training run; returns per-round arrays: loss (mean over workers), T_round, backups (mean b)."""
+        lagged: bool = False, **overrides) -> Dict[str, np.ndarray]:
+    """One training run; returns per-round arrays: loss (mean over workers), T_round, backups (mean b).
+
+    `lagged`: the backup counts of iteration k come from the arrival times of iteration k-1 (set after
+    that iteration, as Algorithm 1 is printed) instead of from the times of the iteration about to run."""
     import torch
     from workloads import configs as wl
     from . import binding as p
@@ -53,7 +56,7 @@ def run(config: int, rounds: Optional[int] = None, dynamic: bool = True, bf16: b
     bs = torch.zeros(rounds, n, dtype=torch.int32, device="cuda")
     for k in range(rounds):
         if dynamic and k > 0:                 # Algorithm 1: the first iteration waits for every neighbour
-            h.update_backups(times[k], b)
+            h.update_backups(times[k - 1] if lagged else times[k], b)
         bs[k].copy_(b)
         h.round(X, times[k], b, wl.learning_rate(w, k), X, kept, batch_idx=dev(wl.batch_indices(w, k)),
                 T_round=Tr[k:k + 1], loss=loss[k])

@@ -149,7 +149,8 @@ def test_mix_matches_oracle(name, d, rule, order):
 
 
 @pytest.mark.parametrize("n,deg,d,order", [(320, 16, 1000, "local_then_mix"), (700, 16, 1300, "mix_then_correct"),
-                                           (1000, 32, 2052, "local_then_mix")])
+                                           (1000, 32, 2052, "local_then_mix"), (512, 8, 516, "local_then_mix"),
+                                           (514, 8, 260, "mix_then_correct")])
 def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
     """The dense 0/1-selection product on the tensor cores (three exact BF16 pieces per fp32 value): worker
     counts that leave ragged row tiles and K chunks, widths that leave a ragged last panel, both update

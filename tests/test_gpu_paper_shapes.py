@@ -17,7 +17,7 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _parity(config, rounds, bf16, tol=1e-5, **overrides):
+def _parity(config, rounds, bf16, tol=1e-5, lagged=False, **overrides):
     import paper_2102_06280_b200 as p
     w = wl.make_workload(config, samples=2048, **overrides)
     m = p.model_layout(w.layers, w.batch)
@@ -41,8 +41,9 @@ def _parity(config, rounds, bf16, tol=1e-5, **overrides):
         t, lr, idx = times[k], wl.learning_rate(w, k), wl.batch_indices(w, k)
         b = np.zeros(w.N, dtype=np.int32)
         if k > 0:
-            b, theta = ref_rule.update_backups(t)
-            h.update_backups(dev(t), b_d, th)
+            t_rule = times[k - 1] if lagged else t                       # lagged: Algorithm 1 read literally
+            b, theta = ref_rule.update_backups(t_rule)
+            h.update_backups(dev(t_rule), b_d, th)
             assert np.array_equal(b_d.cpu().numpy(), b) and float(th.cpu()[0]) == theta
         start = X_ref if bf16 else X_ref.astype(np.float32)          # fp32: teacher-forced every round
         r = orc.dbw_round(w.rowptr, w.col, start, t, b, lr, layers=w.layers,
@@ -53,7 +54,7 @@ def _parity(config, rounds, bf16, tol=1e-5, **overrides):
         torch.cuda.synchronize()
         assert np.array_equal(kept.cpu().numpy(), r["kept"])
         assert np.array_equal(Tw.cpu().numpy(), r["T_worker"]) and float(Tr.cpu()[0]) == r["T_round"]
-        if k > 0:
+        if k > 0 and not lagged:
             assert r["T_round"] == theta                                 # the iteration lasts exactly theta
         got = m.unpack(out.cpu().numpy()).astype(np.float64)
         if not bf16:
@@ -85,6 +86,19 @@ def test_2nn_10_workers_bf16_20_rounds():
     # two free-running trajectories separate, so that schedule is only run for three rounds
     _parity(6, 20, bf16=True, tol=2e-3, lr=0.05)
     _parity(6, 3, bf16=True, tol=2e-2)
+
+
+def test_non_iid_shards_fp32_parity():
+    """Every worker holds two of the ten classes (its own distribution D_j): same parity bars."""
+    _parity(5, 5, bf16=False, label_skew=2)
+
+
+def test_lagged_backup_counts_parity():
+    """b(k) set after iteration k-1 from that iteration's arrival times (Algorithm 1 taken literally)
+    instead of from the times of the iteration about to run: kept masks are no longer symmetric and an
+    iteration no longer lasts exactly theta, but masks, times, b and theta still match bit for bit."""
+    _parity(5, 6, bf16=False, lagged=True)
+    _parity(6, 4, bf16=False, lagged=True, lr=0.05)       # eta_0 = 1 would need the looser bar of the test above
 
 
 @pytest.mark.parametrize("config", [5, 6])

@@ -421,3 +421,21 @@ def test_per_link_times_brute_force_and_reduction():
             assert np.array_equal(a0[0], a1[0]) and np.array_equal(a0[1], a1[1]) and a0[2] == a1[2]
             assert a0[2] == (t[(deg - b >= 1) | np.isin(np.arange(n), col[k0 == 1])].max()
                              if ((deg - b >= 1).any() or k0.any()) else 0.0)
+
+
+def test_non_iid_shards_hold_only_their_classes():
+    """Input recipe: with label_skew = k worker i draws labels from classes (i*k + 0..k-1) mod 10 only, and the
+    features still are class mean + noise (the label decides the mean)."""
+    w = wl.make_workload(5, samples=512, label_skew=2)
+    means = wl.class_means(w)
+    seen = set()
+    for i in range(w.N):
+        f, l = wl.worker_dataset(w, i, means)
+        own = {(2 * i) % 10, (2 * i + 1) % 10}
+        assert set(np.unique(l)) <= own and len(set(np.unique(l))) == 2
+        seen |= own
+        resid = f - means[l]
+        assert abs(float(resid.std()) - w.noise) < 0.05
+    assert len(seen) == 10
+    f0, l0 = wl.worker_dataset(wl.make_workload(5, samples=512), 0, means)
+    assert len(np.unique(l0)) == 10

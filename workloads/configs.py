@@ -170,6 +170,7 @@ class Workload:
     noise: float = 0.0
     clip: bool = False
     means_seed: int = 0
+    label_skew: int = 0              # 0: labels uniform over all classes (iid shards); k > 0: worker i only holds k classes
     batch: int = 0
     lr: float = 0.05
     lr_decay: float = 1.0            # eta(k) = lr * lr_decay^k (k = 0 for the first round)
@@ -267,12 +268,19 @@ def worker_dataset(w: Workload, i: int, means: Optional[np.ndarray] = None):
     """Worker i's shard: features (samples, in) float32, labels (samples,) int32.
 
     feature = mean[label] + noise * N(0,1), clipped to [0,1] for the
-    MNIST-shaped configs; labels uniform over the classes.
+    MNIST-shaped configs; labels uniform over the classes, or, with
+    `label_skew` = k > 0, over the k classes (i*k + 0..k-1) mod classes only
+    (non-iid shards: every worker sees its own D_j).
     """
     if means is None:
         means = class_means(w)
     rng = _rng(_seed(w.index, "data"), i)
-    labels = rng.integers(0, w.layers[-1], size=w.samples).astype(np.int32)
+    classes = w.layers[-1]
+    if w.label_skew > 0:
+        own = (i * w.label_skew + np.arange(w.label_skew)) % classes
+        labels = own[rng.integers(0, w.label_skew, size=w.samples)].astype(np.int32)
+    else:
+        labels = rng.integers(0, classes, size=w.samples).astype(np.int32)
     feats = rng.standard_normal((w.samples, w.layers[0]), dtype=np.float32)
     feats *= np.float32(w.noise)
     feats += means[labels]
