@@ -380,18 +380,33 @@ __global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ l
     }
 }
 
-// db[o] = sum over the batch of dZ[s][o] (dZ bf16 [B][out]); thread per output, coalesced across o.
-__global__ void __launch_bounds__(128)
+// db[o] = sum over the batch of dZ[s][o] (dZ bf16 [B][out], out even).  A block of 256 threads owns 128
+// outputs: a thread sums two adjacent outputs (one 32-bit load per sample) over every fourth sample,
+// and the four partial sums are added through shared memory in a fixed order.
+__global__ void __launch_bounds__(256)
 bias_grad_bf16_kernel(int out_dim, int B, const bf16* __restrict__ dz, long long dz_z, float* __restrict__ G, long long ld,
                       long long b_off) {
+    __shared__ float2 part[4][64];
     const int i = blockIdx.y;
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= out_dim) return;
-    const bf16* p = dz + (size_t)i * dz_z + o;
-    float s = 0.f;
+    const int pair = threadIdx.x & 63, slice = threadIdx.x >> 6;
+    const int o = blockIdx.x * 128 + 2 * pair;
+    float2 s = make_float2(0.f, 0.f);
+    if (o < out_dim) {
+        const bf16* p = dz + (size_t)i * dz_z + o;
 #pragma unroll 8
-    for (int m = 0; m < B; ++m) s += __bfloat162float(p[(size_t)m * out_dim]);
-    G[(size_t)i * ld + b_off + o] = s;
+        for (int m = slice; m < B; m += 4) {
+            const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(p + (size_t)m * out_dim));
+            s.x += __uint_as_float(v << 16);
+            s.y += __uint_as_float(v & 0xffff0000u);
+        }
+    }
+    part[slice][pair] = s;
+    __syncthreads();
+    if (slice == 0 && o < out_dim) {
+        const float2 a = part[0][pair], b = part[1][pair], c = part[2][pair], d = part[3][pair];
+        G[(size_t)i * ld + b_off + o] = ((a.x + b.x) + c.x) + d.x;
+        G[(size_t)i * ld + b_off + o + 1] = ((a.y + b.y) + c.y) + d.y;
+    }
 }
 
 // ----------------------------------------------------------------------------- last layer on CUDA cores
@@ -808,7 +823,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
     if (C <= 16)
-        head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+        head_forward_kernel<16, 4><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     else
         head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
@@ -838,7 +853,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         w.outf = G + m.w_off[l]; w.outf_z = h->ld; w.outf_pitch = in;
         w.status = h->d_status;
         if ((rc = run_tc(st->dwA[l], st->dwB[l], w, N, s, true, true))) return rc;
-        bias_grad_bf16_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(out, B, st->dZ[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
+        bias_grad_bf16_kernel<<<dim3((out + 127) / 128, N), 256, 0, s>>>(out, B, st->dZ[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
         DBW_LAUNCHED();
         if (l >= 1) {
             TcArgs a{};
