@@ -777,6 +777,7 @@ int grad_bf16_alloc(dbw_handle* h) {
         }
     }
     if (!ok) return DBW_ERR_CUDA;
+    DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     return DBW_OK;
@@ -835,7 +836,10 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     }
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
     const int parts = B >= 64 ? 4 : 1;
-    if (C <= 16)
+    if (C <= 12)  // ten classes: a quarter fewer multiply-adds than with the 16-class instance
+        head_backward_kernel<12, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 12 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
+    else if (C <= 16)
         head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
             B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
     else
