@@ -85,20 +85,20 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
     }
 }
 
-// Fallback for graphs too large for a shared-memory panel: one thread per 4 output columns,
-// neighbour rows re-read through L2.  Out of place only.
+// Fallback for graphs too large for a shared-memory panel: neighbour rows are re-read through L2.
+// A work item is one output row of one column panel; a block computes it with consecutive lanes on
+// consecutive columns (every neighbour read of a warp is one contiguous 512-byte segment).  Items are
+// numbered row-fastest inside a panel and handed out in order, so the blocks that run at the same
+// time work on the same column panel, whose X and G segments (N x panel_cols x 8 bytes, sized to sit
+// in L2) are fetched from HBM once and re-read out of L2 by the rows that keep them.  Out of place only.
 __global__ void __launch_bounds__(256)
 mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float* __restrict__ G, float lr,
                   const float* __restrict__ lr_pw, float* __restrict__ Xout, uint16_t* __restrict__ shadow,
-                  MixPlan plan, int mix_then_correct) {
-    const long long ld4 = ld / 4;
-    const long long total = (long long)N * ld4;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
-         e += (long long)gridDim.x * blockDim.x) {
-        // consecutive threads walk down the rows of one column group so that neighbour reads of
-        // concurrently running threads fall in the same few columns (L2 reuse)
-        const int i = (int)(e % N);
-        const long long c = 4 * (e / N);
+                  MixPlan plan, int mix_then_correct, int panel_cols, long long n_items) {
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int i = (int)(item % N);
+        const long long c = (item / N) * panel_cols + 4 * (long long)threadIdx.x;
+        if (c >= ld) continue;
         auto stepped = [&](int r) {
             float4 v = ldg4(X + (size_t)r * ld + c);
             if (!mix_then_correct) v = fma4(-(lr_pw ? lr_pw[r] : lr), ldg4(G + (size_t)r * ld + c), v);
@@ -108,8 +108,17 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
         const float4 self = stepped(i);
         float4 acc = make_float4(ws * self.x, ws * self.y, ws * self.z, ws * self.w);
         const int cnt = plan.cnt[i];
-        for (int k = 0; k < cnt; ++k)
-            acc = fma4(plan.w[(size_t)i * plan.stride + k], stepped(plan.idx[(size_t)i * plan.stride + k]), acc);
+        const int* pi = plan.idx + (size_t)i * plan.stride;
+        const float* pw = plan.w + (size_t)i * plan.stride;
+        int k = 0;
+        for (; k + 4 <= cnt; k += 4) {  // four neighbour rows in flight, added in list order
+            const float4 v0 = stepped(pi[k]), v1 = stepped(pi[k + 1]), v2 = stepped(pi[k + 2]), v3 = stepped(pi[k + 3]);
+            acc = fma4(pw[k], v0, acc);
+            acc = fma4(pw[k + 1], v1, acc);
+            acc = fma4(pw[k + 2], v2, acc);
+            acc = fma4(pw[k + 3], v3, acc);
+        }
+        for (; k < cnt; ++k) acc = fma4(pw[k], stepped(pi[k]), acc);
         if (mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
         *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
         if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
@@ -182,12 +191,15 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
         default: break;
     }
     if (X_out == X) return DBW_ERR_BAD_SHAPE;
-    const long long total = (long long)h->N * (h->ld / 4);
-    long long blocks = (total + 255) / 256;
-    const long long cap = (long long)h->sm_count * 8;
-    if (blocks > cap) blocks = cap;
-    mix_direct_kernel<<<(int)blocks, 256, 0, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, shadow, h->plan,
-                                                 (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0);
+    // panel width: the widest of 1024 / 512 / 256 / 128 columns whose X and G segments of all rows fit in
+    // 48 MB (well inside L2), and no wider than the matrix
+    int panel_cols = 1024;
+    while (panel_cols > 128 && ((long long)h->N * panel_cols * 8 > (48ll << 20) || panel_cols / 2 >= h->ld)) panel_cols >>= 1;
+    const long long n_items = ((h->ld + panel_cols - 1) / panel_cols) * h->N;
+    long long blocks = (long long)h->sm_count * (2048 / (panel_cols / 4) > 16 ? 16 : 2048 / (panel_cols / 4));
+    if (blocks > n_items) blocks = n_items;
+    mix_direct_kernel<<<(int)blocks, panel_cols / 4, 0, s>>>(h->N, h->ld, X, G, lr, lr_pw, X_out, shadow, h->plan,
+                                                           (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0, panel_cols, n_items);
     DBW_LAUNCHED();
     return DBW_OK;
 }

@@ -367,9 +367,12 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
                     if (!plain) {
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
-                        if (lane == 0 && row0 < a.N && colb < a.ld) {
-                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                                         ::"l"(&tmOut), "r"((int)colb), "r"(row0), "r"(smem_u32(buf)) : "memory");
+                        if (lane == 0) {
+                            if (row0 < a.N && colb < a.ld)
+                                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                             ::"l"(&tmOut), "r"((int)colb), "r"(row0), "r"(smem_u32(buf)) : "memory");
+                            // one group per block, empty or not: "at most one group pending" above then always means
+                            // that the store which last read THIS buffer, two blocks ago, is done with it
                             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
                     } else {

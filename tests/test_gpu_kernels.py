@@ -197,6 +197,36 @@ def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
     h.close()
 
 
+def test_mix_large_worker_count_uses_the_l2_kernel():
+    """More workers than a shared-memory panel of even 16 columns can hold: neighbour rows are re-read through L2
+    (row-fastest work order inside column panels), out of place only, same bar."""
+    p = _dbw()
+    n, d = 4200, 1100
+    rowptr, col = wl.random_regular(n, 4, 5)
+    deg = np.diff(rowptr)
+    for rule, order in (("metropolis", "local_then_mix"), ("uniform", "mix_then_correct")):
+        flags = (p.WEIGHT_UNIFORM if rule == "uniform" else 0) | (p.ORDER_MIX_THEN_CORRECT if order == "mix_then_correct" else 0)
+        h = p.Dbw(rowptr, col, d=d, ld=d, flags=flags)
+        assert h.mix_kernel() == "mix_direct_kernel" and not h.mix_in_place_ok()
+        rng = np.random.default_rng(3)
+        X = rng.standard_normal((n, d), dtype=np.float32)
+        G = rng.standard_normal((n, d), dtype=np.float32)
+        t = 1.0 + rng.exponential(1.0, size=n)
+        b = rng.integers(0, deg + 1)
+        kept = orc.select_fastest(rowptr, col, t, b)
+        ws, we = orc.mixing_weights(rowptr, col, b, kept, rule)
+        ref = orc.mix_update(rowptr, col, X, G, ws, we, 0.05, order)
+        Xd = dev(X)
+        out = torch.full_like(Xd, float("nan"))
+        h.mix(Xd, dev(G), dev(kept), dev(b.astype(np.int32)), 0.05, out)
+        torch.cuda.synchronize()
+        assert row_rel_err(out.cpu().numpy(), ref) <= 1e-5
+        with pytest.raises(p.DbwError):
+            h.mix(Xd, dev(G), dev(kept), dev(b.astype(np.int32)), 0.05, Xd)
+        assert h.status() == 0
+        h.close()
+
+
 def test_mix_rejects_bad_aliasing():
     p = _dbw()
     rowptr, col = wl.ring(8)
