@@ -1,4 +1,4 @@
-// Mix kernel for many workers and many terms per output (uniform weights): one persistent CTA per
+// Mix kernel for many workers and many terms per output: one persistent CTA per
 // SM, warp-specialised, with the NEXT column panel prefetched into tensor memory.
 //
 // With N of the order of 1000 a 32-column panel of all rows (N x 128 B) plus the neighbour lists
@@ -9,8 +9,9 @@
 // warps gather the current panel out of shared memory (the gather waits on shared-memory round
 // trips, so it wants every warp the SM can hold).  When both are done the producers move the parked
 // panel from tensor memory into shared memory (tcgen05.ld + 128-bit shared stores) and the roles
-// repeat.  The neighbour lists (16-bit indices, built once per launch from the mixing plan) stay in
-// shared memory for the whole launch.  HBM traffic is the algorithmic 12 bytes per element; a panel
+// repeat.  The neighbour lists (16-bit entries built once per launch from the mixing plan: a bare row
+// index with uniform weights, a 10-bit index and a 6-bit weight code with the Metropolis weights) stay
+// in shared memory for the whole launch.  HBM traffic is the algorithmic 12 bytes per element; a panel
 // is fully staged before any of it is written and panels are disjoint, so X' may overwrite X.
 #include "common.cuh"
 
@@ -22,6 +23,17 @@ constexpr int kProdWarps = 8, kConsWarps = 24;
 constexpr int kThreads = (kProdWarps + kConsWarps) * 32;  // 1024
 constexpr int kTmemCols = 256;                            // 128 lanes x 256 columns x 4 B = one 1024 x 32 panel
 constexpr int kMaxN = 1024;
+constexpr int kZeroCode = 63;  // weight code of list padding (weighted lists): weight 0
+
+// 1 / (1 + m) for the weight codes m = 0 .. 62 of the weighted lists (Assumption 1: the weight worker i puts on a kept
+// neighbour j is 1 / (1 + max(p_i, p_j))), the same fp32 quotient the mixing plan holds; code 63 is weight 0.
+__constant__ float c_weight[64] = {
+    1.0f / 1,  1.0f / 2,  1.0f / 3,  1.0f / 4,  1.0f / 5,  1.0f / 6,  1.0f / 7,  1.0f / 8,  1.0f / 9,  1.0f / 10, 1.0f / 11,
+    1.0f / 12, 1.0f / 13, 1.0f / 14, 1.0f / 15, 1.0f / 16, 1.0f / 17, 1.0f / 18, 1.0f / 19, 1.0f / 20, 1.0f / 21, 1.0f / 22,
+    1.0f / 23, 1.0f / 24, 1.0f / 25, 1.0f / 26, 1.0f / 27, 1.0f / 28, 1.0f / 29, 1.0f / 30, 1.0f / 31, 1.0f / 32, 1.0f / 33,
+    1.0f / 34, 1.0f / 35, 1.0f / 36, 1.0f / 37, 1.0f / 38, 1.0f / 39, 1.0f / 40, 1.0f / 41, 1.0f / 42, 1.0f / 43, 1.0f / 44,
+    1.0f / 45, 1.0f / 46, 1.0f / 47, 1.0f / 48, 1.0f / 49, 1.0f / 50, 1.0f / 51, 1.0f / 52, 1.0f / 53, 1.0f / 54, 1.0f / 55,
+    1.0f / 56, 1.0f / 57, 1.0f / 58, 1.0f / 59, 1.0f / 60, 1.0f / 61, 1.0f / 62, 1.0f / 63, 0.0f};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -49,6 +61,9 @@ __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpre
 __device__ __forceinline__ void add4(float4& a, const float4 v) {
     a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
 }
+__device__ __forceinline__ void fma4(float4& a, const float w, const float4 v) {
+    a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y); a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+}
 
 struct StagedArgs {
     int N, n_panels, mix_then_correct, plan_row;  // plan_row: 16-bit entries per neighbour-list row (multiple of 8)
@@ -65,6 +80,9 @@ struct StagedArgs {
 // Shared memory: panel float4 [N + 1][8] (row N is all zero: the target of list padding), then the
 // neighbour lists uint16 [N][plan_row + 8] (the 16-byte skew keeps four consecutive rows in distinct
 // banks), then the per-row scale float [N], then the list lengths in blocks of 8, uint8 [N].
+// WEIGHTED = false: uniform weights, a list entry is a bare 16-bit row index and the sum is scaled once per row.
+// WEIGHTED = true: a list entry is a 10-bit row index and a 6-bit weight code; padding is (own row, weight 0).
+template <bool WEIGHTED>
 __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
     extern __shared__ float4 smem4[];
     float4* panel = smem4;
@@ -88,9 +106,14 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
             const int k = k0 + 2 * h;
-            const uint32_t lo = k < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + k] : (uint32_t)N;
-            const uint32_t hi = k + 1 < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + k + 1] : (uint32_t)N;
-            w[h] = lo | (hi << 16);
+            auto entry = [&](int kk) -> uint32_t {
+                if (!WEIGHTED) return kk < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + kk] : (uint32_t)N;
+                if (kk >= cnt) return (uint32_t)i | ((uint32_t)kZeroCode << 10);
+                // the plan's weight is 1 / (1 + m): recover m (exact for m <= 62) and keep it as the code
+                const int m = __float2int_rn(1.0f / a.plan.w[(size_t)i * a.plan.stride + kk]) - 1;
+                return (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + kk] | ((uint32_t)min(max(m, 0), kZeroCode - 1) << 10);
+            };
+            w[h] = entry(k) | (entry(k + 1) << 16);
         }
         *reinterpret_cast<uint4*>(lists + (size_t)i * prow + k0) = make_uint4(w[0], w[1], w[2], w[3]);
     }
@@ -165,7 +188,15 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
         const uint4* lp = reinterpret_cast<const uint4*>(lists + (size_t)i * prow);
         int nb = max((int)nblk[i], 1), kb = 0;  // a row without kept neighbours gathers one all-padding block
         uint4 u = lp[0];
-        float4 acc = panel[(size_t)i * 8 + slot];
+        auto first = [&](int row) {  // uniform: the own row, scaled with the sum at the end; weighted: own weight x own row
+            float4 v = panel[(size_t)row * 8 + slot];
+            if (WEIGHTED) {
+                const float ws = scale[row];
+                v.x *= ws; v.y *= ws; v.z *= ws; v.w *= ws;
+            }
+            return v;
+        };
+        float4 acc = first(i);
         while (true) {
             const bool last = kb + 1 >= nb;
             const int i2 = i + kConsWarps * 4;
@@ -174,20 +205,30 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
             uint4 un = u;
             float4 acc2 = acc;
             if (more) un = lp2[last ? 0 : kb + 1];
-            if (last && i2 < N) acc2 = panel[(size_t)i2 * 8 + slot];
-            const float4 v0 = panel[(size_t)(u.x & 0xffffu) * 8 + slot], v1 = panel[(size_t)(u.x >> 16) * 8 + slot];
-            const float4 v2 = panel[(size_t)(u.y & 0xffffu) * 8 + slot], v3 = panel[(size_t)(u.y >> 16) * 8 + slot];
-            const float4 v4 = panel[(size_t)(u.z & 0xffffu) * 8 + slot], v5 = panel[(size_t)(u.z >> 16) * 8 + slot];
-            const float4 v6 = panel[(size_t)(u.w & 0xffffu) * 8 + slot], v7 = panel[(size_t)(u.w >> 16) * 8 + slot];
-            add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
-            add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
+            if (last && i2 < N) acc2 = first(i2);
+            constexpr uint32_t kIdx = WEIGHTED ? 0x3ffu : 0xffffu;
+            const float4 v0 = panel[(size_t)(u.x & kIdx) * 8 + slot], v1 = panel[(size_t)((u.x >> 16) & kIdx) * 8 + slot];
+            const float4 v2 = panel[(size_t)(u.y & kIdx) * 8 + slot], v3 = panel[(size_t)((u.y >> 16) & kIdx) * 8 + slot];
+            const float4 v4 = panel[(size_t)(u.z & kIdx) * 8 + slot], v5 = panel[(size_t)((u.z >> 16) & kIdx) * 8 + slot];
+            const float4 v6 = panel[(size_t)(u.w & kIdx) * 8 + slot], v7 = panel[(size_t)((u.w >> 16) & kIdx) * 8 + slot];
+            if (!WEIGHTED) {
+                add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
+                add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
+            } else {  // weights out of the constant bank (not through the shared-memory pipe), list order
+                fma4(acc, c_weight[(u.x >> 10) & 63u], v0); fma4(acc, c_weight[u.x >> 26], v1);
+                fma4(acc, c_weight[(u.y >> 10) & 63u], v2); fma4(acc, c_weight[u.y >> 26], v3);
+                fma4(acc, c_weight[(u.z >> 10) & 63u], v4); fma4(acc, c_weight[u.z >> 26], v5);
+                fma4(acc, c_weight[(u.w >> 10) & 63u], v6); fma4(acc, c_weight[u.w >> 26], v7);
+            }
             u = un;
             if (!last) {
                 ++kb;
                 continue;
             }
-            const float w = scale[i];
-            acc.x *= w; acc.y *= w; acc.z *= w; acc.w *= w;
+            if (!WEIGHTED) {
+                const float w = scale[i];
+                acc.x *= w; acc.y *= w; acc.z *= w; acc.w *= w;
+            }
             if (c < a.ld) {
                 if (a.mix_then_correct) {
                     const float4 gi = ldg4(a.G + (size_t)i * a.ld + c);
@@ -244,12 +285,12 @@ size_t staged_smem(const dbw_handle* h, int plan_row) {
 
 }  // namespace
 
-// Usable when the weights are uniform (one scale per row, so a list entry is a bare 16-bit index),
-// every worker's panel row fits the tensor-memory staging area, and the shared memory holds panel
-// and lists.
+// Usable when every worker's panel row fits the tensor-memory staging area and the shared memory holds
+// panel and lists; with uniform weights a list entry is a bare 16-bit index (one scale per row), with
+// the Metropolis weights it carries a 6-bit weight code next to a 10-bit index (degrees up to 62).
 bool mix_staged_usable(const dbw_handle* h) {
-    if (!(h->flags & DBW_WEIGHT_UNIFORM)) return false;
     if (h->N > kMaxN || h->N < 64) return false;
+    if (!(h->flags & DBW_WEIGHT_UNIFORM) && h->maxdeg > kZeroCode - 1) return false;
     const int plan_row = (h->maxdeg + 7) / 8 * 8;
     if (plan_row > 248) return false;
     return staged_smem(h, plan_row) + 256 <= (size_t)h->smem_optin;
@@ -267,11 +308,15 @@ int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, c
     const size_t smem = staged_smem(h, a.plan_row);
     static bool configured[64] = {};
     if (!configured[h->device & 63]) {
-        DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
+        DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
+        DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
         configured[h->device & 63] = true;
     }
     const int grid = a.n_panels < h->sm_count ? a.n_panels : h->sm_count;
-    mix_staged_kernel<<<grid, kThreads, smem, s>>>(a);
+    if (h->flags & DBW_WEIGHT_UNIFORM)
+        mix_staged_kernel<false><<<grid, kThreads, smem, s>>>(a);
+    else
+        mix_staged_kernel<true><<<grid, kThreads, smem, s>>>(a);
     DBW_LAUNCHED();
     return DBW_OK;
 }

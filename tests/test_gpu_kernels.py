@@ -197,6 +197,46 @@ def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
     h.close()
 
 
+@pytest.mark.parametrize("order", ["local_then_mix", "mix_then_correct"])
+def test_mix_staged_kernel_with_metropolis_weights(order):
+    """The paper's weight rule (Assumption 1) on a graph with many kept neighbours per worker: the persistent
+    tensor-memory staged kernel is selected by itself, carries the weights as 6-bit codes in its neighbour lists,
+    and adds in the same order as the shared-memory panel kernel: same bits, same bar against the oracle."""
+    p = _dbw()
+    n, deg, d = 1000, 32, 2052
+    rowptr, col = wl.random_regular(n, deg, 7)
+    degs = np.diff(rowptr)
+    h = p.Dbw(rowptr, col, d=d, ld=d, flags=p.ORDER_MIX_THEN_CORRECT if order == "mix_then_correct" else 0)
+    assert h.mix_kernel() == "mix_staged_kernel" and h.mix_in_place_ok()
+    rng = np.random.default_rng(2)
+    X = rng.standard_normal((n, d), dtype=np.float32)
+    G = rng.standard_normal((n, d), dtype=np.float32)
+    t = 1.0 + rng.exponential(1.0, size=n)
+    b = rng.integers(0, np.minimum(degs, 9) + 1)
+    b[0], b[1] = degs[0], 0
+    kept = orc.select_fastest(rowptr, col, t, b)
+    ws, we = orc.mixing_weights(rowptr, col, b, kept, "metropolis")
+    ref = orc.mix_update(rowptr, col, X, G, ws, we, 0.05, order)
+    Xd, Gd, kd, bd = dev(X), dev(G), dev(kept), dev(b.astype(np.int32))
+    res = {}
+    for panel in (0, 16):
+        h.set_mix_panel(panel)
+        out = torch.full_like(Xd, float("nan"))
+        h.mix(Xd, Gd, kd, bd, 0.05, out)
+        torch.cuda.synchronize()
+        res[panel] = out.cpu().numpy()
+        assert row_rel_err(res[panel], ref) <= 1e-5, panel
+    assert h.mix_kernel() == "mix_panel_kernel"
+    assert np.array_equal(res[0], res[16])
+    h.set_mix_panel(0)
+    inpl = Xd.clone()
+    h.mix(inpl, Gd, kd, bd, 0.05, inpl)
+    torch.cuda.synchronize()
+    assert np.array_equal(inpl.cpu().numpy(), res[0])
+    assert h.status() == 0
+    h.close()
+
+
 def test_mix_large_worker_count_uses_the_l2_kernel():
     """More workers than a shared-memory panel of even 16 columns can hold: neighbour rows are re-read through L2
     (row-fastest work order inside column panels), out of place only, same bar."""
