@@ -89,8 +89,8 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
 // A work item is one output row of one column panel; a block computes it with consecutive lanes on
 // consecutive columns (every neighbour read of a warp is one contiguous 512-byte segment).  Items are
 // numbered row-fastest inside a panel and handed out in order, so the blocks that run at the same
-// time work on the same column panel, whose X and G segments (N x panel_cols x 8 bytes, sized to sit
-// in L2) are fetched from HBM once and re-read out of L2 by the rows that keep them.  Out of place only.
+// time work on the same column panel, whose X and G segments (N x panel_cols x 8 bytes, sized to a
+// small share of L2) are fetched from HBM once and re-read out of L2 by the rows that keep them.  Out of place only.
 __global__ void __launch_bounds__(256)
 mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float* __restrict__ G, float lr,
                   const float* __restrict__ lr_pw, float* __restrict__ Xout, uint16_t* __restrict__ shadow,
@@ -191,10 +191,11 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
         default: break;
     }
     if (X_out == X) return DBW_ERR_BAD_SHAPE;
-    // panel width: the widest of 1024 / 512 / 256 / 128 columns whose X and G segments of all rows fit in
-    // 48 MB (well inside L2), and no wider than the matrix
+    // panel width: the widest of 1024 / 512 / 256 columns whose X and G segments of all rows stay within
+    // 12 MB (measured: a small share of L2 keeps the re-reads hitting while the rest of the grid streams
+    // through; 128-column panels leave too few threads per block), and no wider than the matrix needs
     int panel_cols = 1024;
-    while (panel_cols > 128 && ((long long)h->N * panel_cols * 8 > (48ll << 20) || panel_cols / 2 >= h->ld)) panel_cols >>= 1;
+    while (panel_cols > 128 && ((panel_cols > 256 && (long long)h->N * panel_cols * 8 > (12ll << 20)) || panel_cols / 2 >= h->ld)) panel_cols >>= 1;
     const long long n_items = ((h->ld + panel_cols - 1) / panel_cols) * h->N;
     long long blocks = (long long)h->sm_count * (2048 / (panel_cols / 4) > 16 ? 16 : 2048 / (panel_cols / 4));
     if (blocks > n_items) blocks = n_items;

@@ -228,12 +228,16 @@ def test_config3_bf16_free_running_20_rounds():
     _free_run_bf16(wl.make_workload(3, N=16, samples=600), 20)
 
 
-def test_config4_reduced_width():
-    """Config 4's graph, backups, weights and value distributions at d = 8192 (+ ragged tail)."""
+@pytest.mark.parametrize("config,kernel", [(4, "mix_staged_kernel"), (7, "mix_staged_kernel"), (8, "mix_direct_kernel")])
+def test_mix_only_workloads_reduced_width(config, kernel):
+    """The mix-only workloads' graphs, backups, weights and value distributions at d = 8192 (+ ragged tail):
+    config 4 (uniform weights), the paper's weights on the same graph, and 4096 workers (L2 kernel, out of place)."""
     import paper_2102_06280_b200 as p
-    w = wl.make_workload(4, d=8192 + 36)
+    w = wl.make_workload(config, d=8192 + 36, rounds=4 if config != 4 else 10)
     n, d = w.N, w.d
-    h = p.Dbw(w.rowptr, w.col, d=d, flags=p.WEIGHT_UNIFORM)
+    uniform = w.weight_rule == "uniform"
+    h = p.Dbw(w.rowptr, w.col, d=d, flags=p.WEIGHT_UNIFORM if uniform else 0)
+    assert h.mix_kernel() == kernel
     X = wl.gaussian_rows(w.init_seed, range(n), d)
     G = wl.gaussian_rows(wl.external_gradient_seed(w), range(n), d, scale=0.01)
     times = wl.arrival_times(w)
@@ -244,13 +248,15 @@ def test_config4_reduced_width():
     Tr = torch.zeros(1, dtype=torch.float64, device="cuda")
     Xref = X.astype(np.float64)
     for k in range(w.rounds):
-        r = orc.dbw_round(w.rowptr, w.col, Xref.astype(np.float32), times[k], bs[k], w.lr, G=G, rule=orc.UNIFORM)
+        r = orc.dbw_round(w.rowptr, w.col, Xref.astype(np.float32), times[k], bs[k], w.lr, G=G,
+                          rule=orc.UNIFORM if uniform else orc.METROPOLIS)
         Xin = dev(Xref.astype(np.float32))
-        h.round(Xin, dev(times[k]), dev(bs[k]), w.lr, Xin, kept, G_ext=Gd, T_worker=Tw, T_round=Tr)
+        Xout = Xin if h.mix_in_place_ok() else torch.empty_like(Xin)
+        h.round(Xin, dev(times[k]), dev(bs[k]), w.lr, Xout, kept, G_ext=Gd, T_worker=Tw, T_round=Tr)
         torch.cuda.synchronize()
         assert np.array_equal(kept.cpu().numpy(), r["kept"])
         assert np.array_equal(Tw.cpu().numpy(), r["T_worker"]) and float(Tr.cpu()[0]) == r["T_round"]
-        assert row_rel_err(Xin.cpu().numpy(), r["X"]) <= 1e-5
+        assert row_rel_err(Xout.cpu().numpy(), r["X"]) <= 1e-5
         Xref = r["X"]
     assert h.status() == 0
     h.close()

@@ -221,6 +221,12 @@ CONFIGS = {
     4: dict(name="c4_reg32_n1024_mix", N=1024, graph="regular", degree=32, layers=None,
             d=1 << 20, rounds=10, backups="uniform", max_b=8, weight_rule="uniform",
             init="gaussian", init_seed=4),
+    # Two more mix-only workloads beyond the five: the paper's own weight rule (Assumption 1) on the graph of
+    # workload 4, and a worker count too large for any shared-memory panel of all rows.
+    7: dict(name="m0_reg32_n1024_metropolis", N=1024, graph="regular", degree=32, graph_seed=5001, layers=None,
+            d=1 << 20, rounds=10, backups="uniform", max_b=8, weight_rule="metropolis", init="gaussian"),
+    8: dict(name="m1_reg8_n4096_metropolis", N=4096, graph="regular", degree=8, layers=None,
+            d=1 << 16, rounds=10, backups="uniform", max_b=2, weight_rule="metropolis", init="gaussian"),
 }
 
 
