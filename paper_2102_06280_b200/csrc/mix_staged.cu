@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
     uint16_t* lists = reinterpret_cast<uint16_t*>(panel + (size_t)(N + 1) * 8);
     float* scale = reinterpret_cast<float*>(lists + (size_t)N * prow);
     uint8_t* nblk = reinterpret_cast<uint8_t*>(scale + N);
+    float* wtab = reinterpret_cast<float*>(nblk + (N + 15) / 16 * 16);  // copy of c_weight (weighted lists)
     __shared__ uint32_t tmem_slot;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -121,6 +122,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
         scale[i] = a.plan.w_self[i];
         nblk[i] = (uint8_t)((a.plan.cnt[i] + 7) / 8);
     }
+    if (WEIGHTED && tid < 64) wtab[tid] = c_weight[tid];
     if (tid < 8) panel[(size_t)N * 8 + tid] = make_float4(0.f, 0.f, 0.f, 0.f);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -214,11 +216,11 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
             if (!WEIGHTED) {
                 add4(acc, v0); add4(acc, v1); add4(acc, v2); add4(acc, v3);
                 add4(acc, v4); add4(acc, v5); add4(acc, v6); add4(acc, v7);
-            } else {  // weights out of the constant bank (not through the shared-memory pipe), list order
-                fma4(acc, c_weight[(u.x >> 10) & 63u], v0); fma4(acc, c_weight[u.x >> 26], v1);
-                fma4(acc, c_weight[(u.y >> 10) & 63u], v2); fma4(acc, c_weight[u.y >> 26], v3);
-                fma4(acc, c_weight[(u.z >> 10) & 63u], v4); fma4(acc, c_weight[u.z >> 26], v5);
-                fma4(acc, c_weight[(u.w >> 10) & 63u], v6); fma4(acc, c_weight[u.w >> 26], v7);
+            } else {  // weights out of a 64-entry table in shared memory (one wavefront for the warp's four codes), list order
+                fma4(acc, wtab[(u.x >> 10) & 63u], v0); fma4(acc, wtab[u.x >> 26], v1);
+                fma4(acc, wtab[(u.y >> 10) & 63u], v2); fma4(acc, wtab[u.y >> 26], v3);
+                fma4(acc, wtab[(u.z >> 10) & 63u], v4); fma4(acc, wtab[u.z >> 26], v5);
+                fma4(acc, wtab[(u.w >> 10) & 63u], v6); fma4(acc, wtab[u.w >> 26], v7);
             }
             u = un;
             if (!last) {
@@ -280,7 +282,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
 
 size_t staged_smem(const dbw_handle* h, int plan_row) {
     const size_t N = (size_t)h->N;
-    return (N + 1) * 128 + N * (size_t)(plan_row + 8) * 2 + N * 4 + ((N + 15) / 16) * 16;
+    return (N + 1) * 128 + N * (size_t)(plan_row + 8) * 2 + N * 4 + ((N + 15) / 16) * 16 + 256;
 }
 
 }  // namespace
