@@ -125,10 +125,11 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 
 // ------------------------------------------------------------------ softmax cross-entropy
 // One CTA per worker, one warp per sample at a time.  dZ = (softmax(z) - onehot(y)) / B;
-// loss = mean over the batch of (logsumexp(z) - z_y), summed in a fixed order.
+// loss = mean over the batch of (logsumexp(z) - z_y), summed in a fixed order.  The CTA then also sums
+// its worker's dZ over the batch: the bias gradient of the last layer (one launch less per round).
 __global__ void __launch_bounds__(256)
 softmax_ce_kernel(int B, int C, const float* __restrict__ logits, const int32_t* __restrict__ ylab,
-                  float* __restrict__ dz, float* __restrict__ loss) {
+                  float* dz, float* __restrict__ loss, float* __restrict__ G, long long ld, long long b_off) {
     const int i = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float invB = 1.0f / (float)B;
@@ -156,6 +157,13 @@ softmax_ce_kernel(int B, int C, const float* __restrict__ logits, const int32_t*
         float t = 0.f;
         for (int w = 0; w < 8; ++w) t += sl[w];
         loss[i] = t * invB;
+    }
+    // db[c] = sum over the samples of dZ[s][c], in sample order (the barrier above ordered the dZ stores)
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        const float* p = dz + (size_t)i * B * C + c;
+        float t = 0.f;
+        for (int s = 0; s < B; ++s) t += p[(size_t)s * C];
+        G[(size_t)i * ld + b_off + c] = t;
     }
 }
 
@@ -226,7 +234,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.M = B; g.N = out; g.K = in; g.relu = l < L - 1;
         if ((rc = run_gemm(g, N, h->sm_count, s)) != DBW_OK) return rc;
     }
-    softmax_ce_kernel<<<N, 256, 0, s>>>(B, m.dims[L], h->d_act[L], h->d_ylab, h->d_dz[L], loss);
+    softmax_ce_kernel<<<N, 256, 0, s>>>(B, m.dims[L], h->d_act[L], h->d_ylab, h->d_dz[L], loss, G, h->ld, m.b_off[L - 1]);
     DBW_LAUNCHED();
     // backward
     for (int l = L - 1; l >= 0; --l) {
@@ -237,8 +245,10 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.C = G + m.w_off[l]; g.sCz = h->ld; g.sCm = in;
         g.M = out; g.N = in; g.K = B;
         if ((rc = run_gemm(g, N, h->sm_count, s)) != DBW_OK) return rc;
-        bias_grad_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(B, out, h->d_dz[l + 1], G, h->ld, m.b_off[l]);
-        DBW_LAUNCHED();
+        if (l < L - 1) {  // the last layer's bias gradient came out of the loss kernel
+            bias_grad_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(B, out, h->d_dz[l + 1], G, h->ld, m.b_off[l]);
+            DBW_LAUNCHED();
+        }
         if (l > 0) {  // dZ_{l}[m][k] = (sum_o dZ_{l+1}[m][o] W_l[o][k]) * [A_l[m][k] > 0]
             GemmArgs a{};
             a.A = h->d_dz[l + 1]; a.sAz = (long long)B * out; a.sAm = out; a.sAk = 1;
