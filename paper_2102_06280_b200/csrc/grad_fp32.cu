@@ -46,11 +46,12 @@ struct GemmArgs {
     int relu;
 };
 
-constexpr int TK = 16;
 
 // 256 threads, each an R x R micro-tile: tiles of 64 x 64 (R = 4) for large outputs, 32 x 32 (R = 2)
-// when the larger tile would leave most SMs idle.
-template <int R>
+// when the larger tile would leave most SMs idle.  TK = depth of one k-step: 16, or 64 for the few-CTA
+// case with a long reduction, where a step costs one global-memory round trip whatever its depth
+// (the order of the additions is the same).
+template <int R, int TK>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
     constexpr int T = 16 * R;        // tile edge
     constexpr int PER = T * TK / 256;  // elements of each operand tile a thread stages
@@ -70,11 +71,11 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 #pragma unroll
         for (int r = 0; r < PER; ++r) {
             const int e = tid + r * 256;
-            const int ka = a_k_fast ? (e & 15) : (e / T);
-            const int ma = a_k_fast ? (e >> 4) : (e % T);
+            const int ka = a_k_fast ? (e % TK) : (e / T);
+            const int ma = a_k_fast ? (e / TK) : (e % T);
             pa[r] = (m0 + ma < g.M && k0 + ka < g.K) ? __ldg(A + (size_t)(m0 + ma) * g.sAm + (size_t)(k0 + ka) * g.sAk) : 0.f;
-            const int kb = b_k_fast ? (e & 15) : (e / T);
-            const int nb = b_k_fast ? (e >> 4) : (e % T);
+            const int kb = b_k_fast ? (e % TK) : (e / T);
+            const int nb = b_k_fast ? (e / TK) : (e % T);
             pb[r] = (n0 + nb < g.N && k0 + kb < g.K) ? __ldg(B + (size_t)(n0 + nb) * g.sBn + (size_t)(k0 + kb) * g.sBk) : 0.f;
         }
     };
@@ -83,8 +84,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 #pragma unroll
         for (int r = 0; r < PER; ++r) {
             const int e = tid + r * 256;
-            As[a_k_fast ? (e & 15) : (e / T)][a_k_fast ? (e >> 4) : (e % T)] = pa[r];
-            Bs[b_k_fast ? (e & 15) : (e / T)][b_k_fast ? (e >> 4) : (e % T)] = pb[r];
+            As[a_k_fast ? (e % TK) : (e / T)][a_k_fast ? (e / TK) : (e % T)] = pa[r];
+            Bs[b_k_fast ? (e % TK) : (e / T)][b_k_fast ? (e / TK) : (e % T)] = pb[r];
         }
         __syncthreads();
         fetch(k0 + TK);  // all zero past the end
@@ -183,10 +184,14 @@ int run_gemm(const GemmArgs& g, int batch, int sm_count, cudaStream_t s) {
     const long long big = (long long)((g.N + 63) / 64) * ((g.M + 63) / 64) * batch;
     if (big >= 4LL * sm_count) {
         dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, batch);
-        gemm_simt_kernel<4><<<grid, 256, 0, s>>>(g);
+        gemm_simt_kernel<4, 16><<<grid, 256, 0, s>>>(g);
     } else {
         dim3 grid((g.N + 31) / 32, (g.M + 31) / 32, batch);
-        gemm_simt_kernel<2><<<grid, 256, 0, s>>>(g);
+        const long long ctas = (long long)grid.x * grid.y * grid.z;
+        if (g.K >= 128 && ctas < 2LL * sm_count)  // few CTAs, long reduction
+            gemm_simt_kernel<2, 64><<<grid, 256, 0, s>>>(g);
+        else
+            gemm_simt_kernel<2, 16><<<grid, 256, 0, s>>>(g);
     }
     DBW_LAUNCHED();
     return DBW_OK;
