@@ -92,10 +92,16 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 #pragma unroll
         for (int kk = 0; kk < TK; ++kk) {
             float av[R], bv[R];
-#pragma unroll
-            for (int i = 0; i < R; ++i) {
-                av[i] = As[kk][ty * R + i];
-                bv[i] = Bs[kk][tx * R + i];
+            if constexpr (R == 4) {  // one 128-bit shared load per operand (rows are 16-byte aligned: T + 4 = 68 floats)
+                const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+                const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+                av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
+                bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+            } else {
+                const float2 a2 = *reinterpret_cast<const float2*>(&As[kk][ty * 2]);
+                const float2 b2 = *reinterpret_cast<const float2*>(&Bs[kk][tx * 2]);
+                av[0] = a2.x; av[1] = a2.y;
+                bv[0] = b2.x; bv[1] = b2.y;
             }
 #pragma unroll
             for (int i = 0; i < R; ++i)
