@@ -824,7 +824,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
     if (C <= 16)
-        head_forward_kernel<16, 4><<<dim3((B + 15) / 16, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+        head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     else
         head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
