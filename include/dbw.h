@@ -181,7 +181,7 @@ int dbw_mix(dbw_handle* h, const float* X, const float* G, const uint8_t* kept, 
             float lr, const float* lr_per_worker, float* X_out, void* stream);
 int dbw_mix_in_place_ok(const dbw_handle* h);
 /* Expert knob: columns per shared-memory panel of the mix kernel: 0 = automatic, 16 / 32 / 64 /
- * 128 = fixed (falls back to the direct kernel when N * cols * 4 bytes exceed shared memory),
+ * 128 / 256 = fixed (falls back to the direct kernel when N * cols * 4 bytes exceed shared memory),
  * 1 = the tensor-memory staged kernel wherever it applies (64 <= N <= 1024; with the Metropolis
  *     weights degrees up to 62),
  * 2 = the tensor-core kernel wherever it applies (uniform weights, 256 <= N <= 1024): the mix as a

@@ -316,7 +316,7 @@ int dbw_mix_kernel(const dbw_handle* h) { return h ? mix_kernel_kind(h) : DBW_ER
 
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols) {
     if (!h) return DBW_ERR_NULL;
-    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 2 || cols == 16 || cols == 32 || cols == 64 || cols == 128)) return DBW_ERR_BAD_SHAPE;
+    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 2 || cols == 16 || cols == 32 || cols == 64 || cols == 128 || cols == 256)) return DBW_ERR_BAD_SHAPE;
     h->mix_panel_cols = cols;
     return DBW_OK;
 }

@@ -129,6 +129,9 @@ int auto_group_size(const dbw_handle* h) {
     if (h->mix_panel_cols < 0) return 0;  // direct kernel forced
     if (h->mix_panel_cols == 1 || h->mix_panel_cols == 2) return 0; // staged / tensor-core kernel forced (handled by the caller)
     if (h->mix_panel_cols) return ((size_t)h->N * h->mix_panel_cols * 4 <= (size_t)h->smem_optin) ? h->mix_panel_cols / 4 : 0;
+    // few workers and a matrix that streams from HBM (well beyond L2): 256-column panels (1 KB row segments) while
+    // three CTAs still share an SM
+    if ((size_t)h->N * 64 * 16 <= (size_t)(h->smem_optin) / 3 - 1024 && (size_t)h->N * h->ld * 4 > ((size_t)256 << 20)) return 64;
     // widest panel whose staging buffer still lets two CTAs share an SM
     const size_t budget = (size_t)(h->smem_optin) / 2 - 1024;
     for (int gs = 32; gs >= 4; gs >>= 1)
@@ -184,6 +187,7 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
     if (use_tc(h)) return launch_mix_tc(h, X, G, lr, lr_pw, X_out, shadow, s);
     if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, shadow, s);
     switch (auto_group_size(h)) {
+        case 64: return launch_panel<64>(h, X, G, lr, lr_pw, X_out, shadow, s);
         case 32: return launch_panel<32>(h, X, G, lr, lr_pw, X_out, shadow, s);
         case 16: return launch_panel<16>(h, X, G, lr, lr_pw, X_out, shadow, s);
         case 8: return launch_panel<8>(h, X, G, lr, lr_pw, X_out, shadow, s);

@@ -123,7 +123,7 @@ def test_mix_matches_oracle(name, d, rule, order):
     ws, we = orc.mixing_weights(rowptr, col, b, kept, rule)
     ref = orc.mix_update(rowptr, col, X, G, ws, we, 0.05, order)
     Xd, Gd, kd, bd = dev(X), dev(G), dev(kept), dev(b.astype(np.int32))
-    for panel in (0, 1, 2, 16, 32, 64, 128, -1):
+    for panel in (0, 1, 2, 16, 32, 64, 128, 256, -1):
         h.set_mix_panel(panel)
         out = torch.full_like(Xd, float("nan"))
         h.mix(Xd, Gd, kd, bd, 0.05, out)
