@@ -196,7 +196,9 @@ int dbw_mix_kernel(const dbw_handle* h);
 /*
  * Algorithm 1, one iteration: gradients (dbw_grad, or G_ext when batch_idx is NULL), selection
  * (dbw_select) and the update (dbw_mix) in one call.  Arguments as in those three; loss is
- * nullable; G_ext [N][ld] is used iff batch_idx == NULL.
+ * nullable; G_ext [N][ld] is used iff batch_idx == NULL.  With batch_idx the selection kernel is
+ * queued on a stream of the handle that waits for everything queued on `stream` so far and that
+ * `stream` waits for before the mix: to the caller all work is still ordered on `stream`.
  */
 int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
               const int32_t* batch_idx, const float* G_ext, float lr, const float* lr_per_worker,
@@ -253,9 +255,11 @@ int dbw_status(dbw_handle* h);
 int dbw_get_links(const dbw_handle* h, int32_t* links);
 
 /*
- * Stage timing.  While enabled, every dbw_round / dbw_round_host records CUDA events on the
- * caller's stream around its stages (0 = gradients, 1 = selection + plan, 2 = mix), up to 4096
- * rounds.  dbw_profile_read() waits for the recorded events, adds their elapsed times to
+ * Stage timing.  While enabled, every dbw_round / dbw_round_host records CUDA events around its
+ * stages (0 = gradients, 1 = selection + plan, 2 = mix), up to 4096 rounds.  When the round computes
+ * gradients the selection, which needs only t and b, runs beside them on a stream of the handle
+ * (forked from and joined back into the caller's stream), so the three times may add up to more
+ * than the round took.  dbw_profile_read() waits for the recorded events, adds their elapsed times to
  * ms[3] (HOST), stores the number of rounds in *rounds and clears the record.  Do not enable
  * it while the stream is being captured into a CUDA graph.
  */

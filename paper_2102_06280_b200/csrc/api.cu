@@ -112,6 +112,11 @@ int dev_alloc(T** p, size_t n) {
 void free_all(dbw_handle* h) {
     for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
     h->prof_events.clear();
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->side) cudaStreamDestroy(h->side);
+    h->ev_fork = h->ev_join = nullptr;
+    h->side = nullptr;
     grad_fp32_free(h);
     grad_bf16_free(h);
     mix_tc_free(h);
@@ -231,6 +236,10 @@ int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* 
               cuda_ok(cudaMemset(h->d_waited, 0, (size_t)N * sizeof(uint32_t))) &&
               cuda_ok(cudaMemset(h->d_ticket, 0, sizeof(uint32_t)));
     if (!ok) return fail(DBW_ERR_CUDA);
+    if (!cuda_ok(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking)) ||
+        !cuda_ok(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) ||
+        !cuda_ok(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)))
+        return fail(DBW_ERR_CUDA);
     if (model) {
         h->has_model = true;
         h->model = *model;
@@ -338,24 +347,38 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
     if ((rc = check_mix_args(h, X, G, X_out))) return rc;
     cudaEvent_t* ev = nullptr;
     if (h->profiling && h->prof_rounds < kProfMaxRounds) {
-        while ((int)h->prof_events.size() < 4 * (h->prof_rounds + 1)) {
+        while ((int)h->prof_events.size() < 6 * (h->prof_rounds + 1)) {
             cudaEvent_t e;
             DBW_CUDA(cudaEventCreate(&e));
             h->prof_events.push_back(e);
         }
-        ev = &h->prof_events[4 * h->prof_rounds++];
-        DBW_CUDA(cudaEventRecord(ev[0], s));
+        ev = &h->prof_events[6 * h->prof_rounds++];
     }
+    // The selection needs only t and b, so with gradients to compute it runs beside them on the handle's
+    // side stream: fork after everything the caller queued, join before the mix.
+    cudaStream_t sel = s;
     if (batch_idx) {
+        sel = h->side;
+        DBW_CUDA(cudaEventRecord(h->ev_fork, s));
+        DBW_CUDA(cudaStreamWaitEvent(sel, h->ev_fork, 0));
+    }
+    if (ev) DBW_CUDA(cudaEventRecord(ev[2], sel));
+    if ((rc = launch_select(h, t, b, kept, T_worker, T_nbr, T_round, true, sel))) return rc;
+    if (ev) DBW_CUDA(cudaEventRecord(ev[3], sel));
+    if (ev) DBW_CUDA(cudaEventRecord(ev[0], s));
+    if (batch_idx) {
+        DBW_CUDA(cudaEventRecord(h->ev_join, sel));
         rc = (h->flags & DBW_GEMM_BF16) ? launch_grad_bf16(h, X, batch_idx, h->d_G, loss, s)
                                         : launch_grad_fp32(h, X, batch_idx, h->d_G, loss, s);
+        if (ev) DBW_CUDA(cudaEventRecord(ev[1], s));
+        DBW_CUDA(cudaStreamWaitEvent(s, h->ev_join, 0));  // joined even when a launch failed: the side stream never dangles
         if (rc) return rc;
+    } else if (ev) {
+        DBW_CUDA(cudaEventRecord(ev[1], s));
     }
-    if (ev) DBW_CUDA(cudaEventRecord(ev[1], s));
-    if ((rc = launch_select(h, t, b, kept, T_worker, T_nbr, T_round, true, s))) return rc;
-    if (ev) DBW_CUDA(cudaEventRecord(ev[2], s));
+    if (ev) DBW_CUDA(cudaEventRecord(ev[4], s));
     rc = launch_mix(h, X, G, lr, lr_per_worker, X_out, s);
-    if (ev) DBW_CUDA(cudaEventRecord(ev[3], s));
+    if (ev) DBW_CUDA(cudaEventRecord(ev[5], s));
     return rc;
 }
 
@@ -369,11 +392,11 @@ int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds) {
     if (!h || !ms || !rounds) return DBW_ERR_NULL;
     DeviceGuard guard(h->device);
     for (int r = 0; r < h->prof_rounds; ++r) {
-        cudaEvent_t* ev = &h->prof_events[4 * r];
-        DBW_CUDA(cudaEventSynchronize(ev[3]));
-        for (int st = 0; st < 3; ++st) {
+        cudaEvent_t* ev = &h->prof_events[6 * r];
+        DBW_CUDA(cudaEventSynchronize(ev[5]));
+        for (int st = 0; st < 3; ++st) {  // gradients, selection (beside the gradients when there are any), mix
             float v = 0.f;
-            DBW_CUDA(cudaEventElapsedTime(&v, ev[st], ev[st + 1]));
+            DBW_CUDA(cudaEventElapsedTime(&v, ev[2 * st], ev[2 * st + 1]));
             ms[st] += v;
         }
     }

@@ -99,7 +99,12 @@ struct dbw_handle {
     bool shadow_valid = false;
     const float* shadow_of = nullptr;
 
-    // stage timing (dbw_profile): events[round][stage boundary 0..3]
+    // selection of dbw_round runs beside the gradient kernels on this stream (forked from and joined back
+    // into the caller's stream by the two events)
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+
+    // stage timing (dbw_profile): events[round][0..5] = start / end of the gradient, selection and mix stages
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;
     int prof_rounds = 0;
