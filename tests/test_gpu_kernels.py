@@ -181,10 +181,11 @@ def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
         torch.cuda.synchronize()
         got = out.cpu().numpy()
         assert row_rel_err(got, ref) <= 1e-5
-        again = torch.empty_like(Xd)
-        h.mix(Xd, Gd, kd, bd, lr, again, lr_per_worker=None if lr_pw is None else dev(lr_pw))
-        torch.cuda.synchronize()
-        assert np.array_equal(again.cpu().numpy(), got)
+        for _ in range(3):                                   # a store racing with the reuse of its staging buffer showed up here once
+            again = torch.zeros_like(Xd)
+            h.mix(Xd, Gd, kd, bd, lr, again, lr_per_worker=None if lr_pw is None else dev(lr_pw))
+            torch.cuda.synchronize()
+            assert np.array_equal(again.cpu().numpy(), got)
         if h.mix_in_place_ok():
             inpl = Xd.clone()
             h.mix(inpl, Gd, kd, bd, lr, inpl, lr_per_worker=None if lr_pw is None else dev(lr_pw))
