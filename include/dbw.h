@@ -56,10 +56,11 @@ enum {
 #define DBW_GEMM_BF16 4u /* dense layers with BF16 operands on tcgen05 tensor cores, fp32 accumulate */
 
 /* bits of the device status word */
-#define DBW_STATUS_BAD_B 1u       /* some b_i was outside [0, deg_i] (clamped) */
+#define DBW_STATUS_BAD_B 1u       /* some b_i was outside [0, deg_i] (clamped), or a kept mask given to dbw_mix
+                                     does not hold deg_i - b_i entries for some i */
 #define DBW_STATUS_NAN_TIME 2u    /* some arrival time was NaN (ordered last) */
 #define DBW_STATUS_WAIT_TIMEOUT 4u /* a bounded pipeline wait expired; results of that call are invalid */
-#define DBW_STATUS_BAD_INDEX 8u   /* a batch index was outside [0, S) (clamped) */
+#define DBW_STATUS_BAD_INDEX 8u   /* a batch index was outside [0, S) or a label outside [0, classes) (clamped) */
 
 #define DBW_MAX_LAYERS 8
 
@@ -171,7 +172,12 @@ int dbw_grad(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, 
 /*
  * Assumption 1 (weights) + Eqs. 4-5 or Eq. 3 (update), every row read from the OLD X.
  * DEVICE in : X [N][ld], G [N][ld], kept[nnz], b[N]; lr scalar; lr_per_worker[N] fp32 nullable
- *             (eta_j; overrides lr).
+ *             (eta_j; overrides lr).  G may be NULL: the gradients are taken as zero and nothing of G
+ *             is read (the consensus-only iterations of the truncated model of Section 3.2.1, whose
+ *             rows converge to their common mean by Corollary 1): 8 bytes per element instead of 12.
+ *             With uniform weights the weight is 1 / (1 + number of entries set in kept's row i); with
+ *             the weights of Assumption 1 the counts p = deg - b of both ends are used.  A row of kept
+ *             that does not hold deg_i - b_i entries sets DBW_STATUS_BAD_B.
  * DEVICE out: X_out [N][ld].  X_out may alias X exactly (in place) when dbw_mix_in_place_ok()
  *             is 1; partial overlap is an error.  G is read only.
  * Summation order per element is fixed (self, then kept neighbours in CSR order), so results
@@ -196,7 +202,8 @@ int dbw_mix_kernel(const dbw_handle* h);
 /*
  * Algorithm 1, one iteration: gradients (dbw_grad, or G_ext when batch_idx is NULL), selection
  * (dbw_select) and the update (dbw_mix) in one call.  Arguments as in those three; loss is
- * nullable; G_ext [N][ld] is used iff batch_idx == NULL.  With batch_idx the selection kernel is
+ * nullable; G_ext [N][ld] is used iff batch_idx == NULL, and when both are NULL the round is a
+ * consensus-only one (G = 0, nothing of G read).  With batch_idx the selection kernel is
  * queued on a stream of the handle that waits for everything queued on `stream` so far and that
  * `stream` waits for before the mix: to the caller all work is still ordered on `stream`.
  */
@@ -265,6 +272,17 @@ int dbw_get_links(const dbw_handle* h, int32_t* links);
  */
 int dbw_profile(dbw_handle* h, int enable);
 int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds);
+
+/*
+ * Self-test of the bounded waits of the tensor-core pipelines (no passage of the paper: a safety
+ * property of this implementation).  Launches one small kernel in which a thread waits, with a limit of
+ * `polls` polls (1 .. 2^20), on a barrier that nothing completes, then waits on it again.  DEVICE
+ * out[3]: out[0] = 1 when the first wait gave up, out[1] = 1 when the second wait returned without
+ * completing, out[2] = clock ticks the second wait took (it must not spin: the first expired wait makes
+ * every later wait of the thread block return at once).  Sets DBW_STATUS_WAIT_TIMEOUT in the handle's
+ * status word, as an expired wait in a real pipeline does; the context stays usable.
+ */
+int dbw_debug_wait_probe(dbw_handle* h, uint32_t polls, uint32_t* out, void* stream);
 
 /* Kernels launched by this library since it was loaded (for launch accounting). */
 int64_t dbw_launch_count(void);

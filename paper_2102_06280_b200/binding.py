@@ -66,6 +66,7 @@ _SIGNATURES = {
     "dbw_get_links": (C.c_int, [_P, _P]),
     "dbw_profile": (C.c_int, [_P, C.c_int]),
     "dbw_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
+    "dbw_debug_wait_probe": (C.c_int, [_P, C.c_uint32, _P, _P]),
     "dbw_launch_count": (C.c_int64, []),
     "dbw_last_cuda_error": (C.c_int, []),
 }
@@ -256,6 +257,9 @@ class Dbw:
         n = C.c_int32(0)
         _check(lib().dbw_profile_read(self._h, ms, C.byref(n)), "dbw_profile_read")
         return {"grad": ms[0], "select": ms[1], "mix": ms[2]}, int(n.value)
+
+    def debug_wait_probe(self, polls: int, out):
+        _check(lib().dbw_debug_wait_probe(self._h, int(polls), _ptr(out), _stream()), "dbw_debug_wait_probe")
 
     def status(self) -> int:
         return _check(lib().dbw_status(self._h), "dbw_status")

@@ -290,20 +290,20 @@ int dbw_grad(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, 
 }
 
 static int check_mix_args(dbw_handle* h, const float* X, const float* G, float* X_out) {
-    if (!aligned16(X) || !aligned16(G) || !aligned16(X_out)) return DBW_ERR_BAD_SHAPE;
+    if (!aligned16(X) || (G && !aligned16(G)) || !aligned16(X_out)) return DBW_ERR_BAD_SHAPE;
     const size_t bytes = (size_t)h->N * h->ld * sizeof(float);
     const char* a = reinterpret_cast<const char*>(X);
     const char* o = reinterpret_cast<const char*>(X_out);
     if (o != a && o < a + bytes && a < o + bytes) return DBW_ERR_BAD_SHAPE;  // partial overlap
     if (o == a && !mix_panel_fits(h)) return DBW_ERR_BAD_SHAPE;
     const char* g = reinterpret_cast<const char*>(G);
-    if (o < g + bytes && g < o + bytes) return DBW_ERR_BAD_SHAPE;  // G is read only
+    if (g && o < g + bytes && g < o + bytes) return DBW_ERR_BAD_SHAPE;  // G is read only
     return DBW_OK;
 }
 
 int dbw_mix(dbw_handle* h, const float* X, const float* G, const uint8_t* kept, const int32_t* b, float lr,
             const float* lr_per_worker, float* X_out, void* stream) {
-    if (!h || !X || !G || !kept || !b || !X_out) return DBW_ERR_NULL;
+    if (!h || !X || !kept || !b || !X_out) return DBW_ERR_NULL;  // G == NULL: consensus only, G = 0
     int rc = check_mix_args(h, X, G, X_out);
     if (rc) return rc;
     DeviceGuard guard(h->device);
@@ -334,11 +334,10 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
               const float* G_ext, float lr, const float* lr_per_worker, float* X_out, uint8_t* kept,
               double* T_worker, double* T_nbr, double* T_round, float* loss, void* stream) {
     if (!h || !X || !t || !b || !X_out || !kept) return DBW_ERR_NULL;
-    if (!batch_idx && !G_ext) return DBW_ERR_NULL;
     DeviceGuard guard(h->device);
     cudaStream_t s = (cudaStream_t)stream;
     int rc;
-    const float* G = G_ext;
+    const float* G = G_ext;  // NULL together with batch_idx == NULL: a consensus-only round, G = 0
     if (batch_idx) {
         if (!h->has_model || !h->feat) return DBW_ERR_BAD_MODEL;
         if ((rc = ensure_G(h))) return rc;
@@ -354,32 +353,40 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
         }
         ev = &h->prof_events[6 * h->prof_rounds++];
     }
+    // first error of the calls below; later calls still run so that a forked side stream is always joined
+    int first = DBW_OK;
+    auto note = [&](int code) {
+        if (first == DBW_OK && code != DBW_OK) first = code;
+    };
+    auto cuda = [&](cudaError_t e) { note(cuda_ok(e) ? DBW_OK : DBW_ERR_CUDA); };
     // The selection needs only t and b, so with gradients to compute it runs beside them on the handle's
     // side stream: fork after everything the caller queued, join before the mix.
     cudaStream_t sel = s;
+    bool forked = false;
     if (batch_idx) {
+        cuda(cudaEventRecord(h->ev_fork, s));
+        if (first == DBW_OK) cuda(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+        if (first != DBW_OK) return first;  // nothing forked yet
         sel = h->side;
-        DBW_CUDA(cudaEventRecord(h->ev_fork, s));
-        DBW_CUDA(cudaStreamWaitEvent(sel, h->ev_fork, 0));
+        forked = true;
     }
-    if (ev) DBW_CUDA(cudaEventRecord(ev[2], sel));
-    if ((rc = launch_select(h, t, b, kept, T_worker, T_nbr, T_round, true, sel))) return rc;
-    if (ev) DBW_CUDA(cudaEventRecord(ev[3], sel));
-    if (ev) DBW_CUDA(cudaEventRecord(ev[0], s));
-    if (batch_idx) {
-        DBW_CUDA(cudaEventRecord(h->ev_join, sel));
-        rc = (h->flags & DBW_GEMM_BF16) ? launch_grad_bf16(h, X, batch_idx, h->d_G, loss, s)
-                                        : launch_grad_fp32(h, X, batch_idx, h->d_G, loss, s);
-        if (ev) DBW_CUDA(cudaEventRecord(ev[1], s));
-        DBW_CUDA(cudaStreamWaitEvent(s, h->ev_join, 0));  // joined even when a launch failed: the side stream never dangles
-        if (rc) return rc;
-    } else if (ev) {
-        DBW_CUDA(cudaEventRecord(ev[1], s));
+    if (ev) cuda(cudaEventRecord(ev[2], sel));
+    note(launch_select(h, t, b, kept, T_worker, T_nbr, T_round, true, sel));
+    if (ev) cuda(cudaEventRecord(ev[3], sel));
+    if (ev) cuda(cudaEventRecord(ev[0], s));
+    if (batch_idx && first == DBW_OK)
+        note((h->flags & DBW_GEMM_BF16) ? launch_grad_bf16(h, X, batch_idx, h->d_G, loss, s)
+                                        : launch_grad_fp32(h, X, batch_idx, h->d_G, loss, s));
+    if (ev) cuda(cudaEventRecord(ev[1], s));
+    if (forked) {  // whatever failed above, the side stream is joined back: it never dangles, a capture stays valid
+        cuda(cudaEventRecord(h->ev_join, sel));
+        cuda(cudaStreamWaitEvent(s, h->ev_join, 0));
     }
-    if (ev) DBW_CUDA(cudaEventRecord(ev[4], s));
-    rc = launch_mix(h, X, G, lr, lr_per_worker, X_out, s);
-    if (ev) DBW_CUDA(cudaEventRecord(ev[5], s));
-    return rc;
+    if (first != DBW_OK) return first;
+    if (ev) cuda(cudaEventRecord(ev[4], s));
+    note(launch_mix(h, X, G, lr, lr_per_worker, X_out, s));
+    if (ev) cuda(cudaEventRecord(ev[5], s));
+    return first;
 }
 
 int dbw_profile(dbw_handle* h, int enable) {
@@ -409,7 +416,6 @@ int dbw_round_host(dbw_handle* h, const float* X, const double* h_t, const int32
                    const int32_t* h_batch_idx, const float* G_ext, float lr, float* X_out, uint8_t* h_kept,
                    double* h_T_worker, double* h_T_round, float* h_loss, int32_t* h_b_out, void* stream) {
     if (!h || !X || !h_t || !X_out) return DBW_ERR_NULL;
-    if (!h_batch_idx && !G_ext) return DBW_ERR_NULL;
     DeviceGuard guard(h->device);
     cudaStream_t s = (cudaStream_t)stream;
     int rc;

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "dbw.h"
@@ -34,6 +35,22 @@ inline bool cuda_ok(cudaError_t e) {
         ::dbw::g_launches.fetch_add(1);                        \
         if (!::dbw::cuda_ok(cudaGetLastError())) return DBW_ERR_CUDA; \
     } while (0)
+
+// One-time set-up per device (kernel attributes, symbol addresses), safe when several host threads
+// make the first call at once: `f` runs under the lock until it has succeeded once on that device.
+struct PerDeviceOnce {
+    std::mutex mu;
+    bool done[64] = {};
+    template <class F>
+    int run(int dev, F&& f) {
+        if (dev < 0 || dev >= 64) return DBW_ERR_BAD_SHAPE;
+        std::lock_guard<std::mutex> lock(mu);
+        if (done[dev]) return DBW_OK;
+        const int rc = f();
+        if (rc == DBW_OK) done[dev] = true;
+        return rc;
+    }
+};
 
 // Per-round mixing plan (built on the device from kept and b): for each worker the compacted
 // list of kept neighbours with their weights, padded to `stride` entries with (self, 0).

@@ -18,6 +18,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace dbw {
 
@@ -26,32 +27,14 @@ namespace {
 typedef __nv_bfloat16 bf16;
 
 // ----------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using namespace ptx;
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: after kSpinLimit failed polls the status word is flagged and the caller goes on,
-// so that every role still reaches the end of the kernel and tensor memory is released.
+// Every mbarrier wait is bounded: after kSpinLimit failed polls the status word is flagged, the CTA's abort
+// word is set and all later waits of the CTA return at once, so that every role still reaches the end of
+// the kernel and tensor memory is released.
 constexpr uint32_t kSpinLimit = 1u << 24;
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return;
-    atomicOr(status, DBW_STATUS_WAIT_TIMEOUT);
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort, uint32_t* status) {
+    return mbar_wait_bounded<false>(bar, parity, kSpinLimit, 0, abort, status);
 }
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
     asm volatile(
@@ -59,8 +42,6 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
         ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
         : "memory");
 }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -72,46 +53,8 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile staged by TMA with the 128-byte swizzle:
-// rows are 128 bytes (64 bf16) apart, groups of 8 rows 1024 bytes apart (stride byte offset),
-// leading byte offset 16 (unused by this layout), descriptor version 1, layout type 2 = 128B.
-__device__ __forceinline__ uint64_t kmajor_sw128_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-
-// MN-major tile (the M or N index is contiguous in memory, K runs over rows) staged by TMA in
-// chunks of 64 (MN) x 64 (K rows) with the 128-byte swizzle: inside a chunk a K row is 128 bytes,
-// groups of 8 K rows are 1024 bytes apart (stride byte offset); chunks along MN follow each other
-// 8192 bytes apart (leading byte offset).
-__device__ __forceinline__ uint64_t mnmajor_sw128_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)(8192 >> 4) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
+// MN-major operand tiles of this file are staged in chunks of 64 (MN) x 64 (K rows): chunks 8192 bytes apart
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t smem_addr) { return mnmajor_sw128_desc(smem_addr, 8192); }
 
 // two floats -> packed bf16x2 (low half = first)
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -145,10 +88,6 @@ struct TcArgs {
     uint32_t* status;
 };
 
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
 constexpr int STAGING_FLOATS = EPI_WARPS * 32 * 36;  // per epilogue warp a 32 x 32 fp32 block, rows 36 words apart
 
 // Persistent, warp-specialised GEMM: one CTA per SM walks the tiles (n fastest, then m, then worker).
@@ -170,12 +109,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;
     uint64_t* acc_empty = acc_full + ACC;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + ACC);
+    uint64_t* drain = acc_empty + ACC;  // shutdown after an expired wait: completion of the MMAs issued so far
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile uint32_t* abort = tmem_slot + 1;  // set by the first wait that runs out; every later wait returns at once
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (g.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
+        *abort = 0u;
+        mbar_init(drain, 1);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
@@ -198,11 +141,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         if (lane == 0) {
             int it = 0;  // k-blocks issued so far, over all tiles of this CTA
-            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            bool live = true;
+            for (int tile = blockIdx.x; tile < n_tiles && live; tile += gridDim.x) {
                 const int n0 = (tile % tiles_n) * BN, m0 = ((tile / tiles_n) % tiles_m) * BM, z = tile / (tiles_n * tiles_m);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
-                    if (it >= STAGES) mbar_wait(&empty[s], ((it / STAGES) - 1) & 1, g.status);
+                    if (it >= STAGES && !mbar_wait(&empty[s], ((it / STAGES) - 1) & 1, abort, g.status)) {
+                        live = false;  // a wait ran out somewhere in this CTA: issue nothing more
+                        break;
+                    }
                     mbar_expect_tx(&full[s], TILE_BYTES + TILE_B_BYTES);
                     if (!AMN) {
                         tma_load_3d(tilesA + s * TILE_BYTES, &tmA, kb * BK, m0, z, &full[s]);
@@ -220,24 +167,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+            // the copies still in flight (the last STAGES at most) have landed before this CTA leaves
+            for (int j = it > STAGES ? it - STAGES : 0; j < it; ++j) mbar_wait_quiet<false>(&full[j % STAGES], (j / STAGES) & 1, 1u << 20);
         }
     } else if (warp == 1) {
         if (lane == 0) {
             int it = 0, lt = 0;
-            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++lt) {
+            bool live = true;
+            for (int tile = blockIdx.x; tile < n_tiles && live; tile += gridDim.x, ++lt) {
                 const int buf = lt % ACC;
                 if (lt >= ACC) {  // the epilogue must have drained this buffer's previous tile
-                    mbar_wait(&acc_empty[buf], ((lt / ACC) - 1) & 1, g.status);
+                    if (!mbar_wait(&acc_empty[buf], ((lt / ACC) - 1) & 1, abort, g.status)) break;
                     tc_fence_after();
                 }
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
-                    mbar_wait(&full[s], (it / STAGES) & 1, g.status);
+                    if (!mbar_wait(&full[s], (it / STAGES) & 1, abort, g.status)) {
+                        live = false;
+                        break;
+                    }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(tilesA + s * TILE_BYTES), sb = smem_u32(tilesB + s * TILE_B_BYTES);
-                    const uint64_t da = AMN ? mnmajor_sw128_desc(sa) : kmajor_sw128_desc(sa);
-                    const uint64_t db = BMN ? mnmajor_sw128_desc(sb) : kmajor_sw128_desc(sb);
+                    const uint64_t da = AMN ? mnmajor_desc(sa) : kmajor_sw128_desc(sa);
+                    const uint64_t db = BMN ? mnmajor_desc(sb) : kmajor_sw128_desc(sb);
                     // 16 further along K: 32 bytes inside the swizzle atom (K-major) or 16 rows of 128 bytes (MN-major)
                     constexpr uint64_t ka = (AMN ? UMMA_K * 128 : UMMA_K * 2) / 16, kbs = (BMN ? UMMA_K * 128 : UMMA_K * 2) / 16;
 #pragma unroll
@@ -245,7 +198,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tc_mma_bf16(d_tmem, da + (uint64_t)k * ka, db + (uint64_t)k * kbs, IDESC, (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit(&empty[s]);  // frees the stage once these MMAs have read it
                 }
-                tc_commit(&acc_full[buf]);
+                if (live) tc_commit(&acc_full[buf]);
+            }
+            if (*abort) {  // shutdown after an expired wait: the MMAs issued so far are complete before tensor memory is freed
+                tc_commit(drain);
+                mbar_wait_quiet<false>(drain, 0, 1u << 20);
             }
         }
     } else {
@@ -258,7 +215,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++lt) {
             const int n0 = (tile % tiles_n) * BN, m0 = ((tile / tiles_n) % tiles_m) * BM, z = tile / (tiles_n * tiles_m);
             const int buf = lt % ACC;
-            mbar_wait(&acc_full[buf], (lt / ACC) & 1, g.status);
+            const bool ready = mbar_wait(&acc_full[buf], (lt / ACC) & 1, abort, g.status);
+            if (!__all_sync(0xffffffffu, ready)) break;  // a wait ran out: leave together (the tensor-memory loads below are warp-collective)
             tc_fence_after();
             const int m = m0 + q * 32 + lane;
             const bool m_ok = m < g.M;
@@ -370,13 +328,20 @@ cast_tile_kernel(int rows, int cols, const float* __restrict__ src, long long sr
     if (c0 + 8 < cols) *reinterpret_cast<uint4*>(d + 8) = pack8(v + 8);
 }
 
-__global__ void gather_labels_kernel(int B, int S, const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
-                                     int32_t* __restrict__ ylab) {
+// Labels of the mini-batch; a label outside [0, C) is clamped and reported (the batch index is
+// reported by the feature gather).
+__global__ void gather_labels_kernel(int B, int S, int C, const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
+                                     int32_t* __restrict__ ylab, uint32_t* status) {
     const int i = blockIdx.x;
     for (int s = threadIdx.x; s < B; s += blockDim.x) {
         int src = batch_idx[(size_t)i * B + s];
         src = src < 0 ? 0 : (src >= S ? S - 1 : src);
-        ylab[(size_t)i * B + s] = labels[(size_t)i * S + src];
+        int y = labels[(size_t)i * S + src];
+        if (y < 0 || y >= C) {
+            atomicOr(status, DBW_STATUS_BAD_INDEX);
+            y = y < 0 ? 0 : C - 1;
+        }
+        ylab[(size_t)i * B + s] = y;
     }
 }
 
@@ -616,26 +581,9 @@ head_reduce_kernel(int B, int K, int C, int parts, int workers, const float* __r
 }
 
 // ----------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // MN-major operand [workers][K rows][MN] bf16 (MN contiguous): box = 64 (MN) x 64 (K rows) x 1.
 bool make_operand_map_mn(CUtensorMap* map, const bf16* base, int MN, int Krows, int workers, long long worker_pitch = 0) {
-    EncodeTiledFn fn = encode_fn();
+    EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     if (!worker_pitch) worker_pitch = (long long)MN * Krows;
     cuuint64_t dims[3] = {(cuuint64_t)MN, (cuuint64_t)Krows, (cuuint64_t)workers};
@@ -651,7 +599,7 @@ bool make_operand_map_mn(CUtensorMap* map, const bf16* base, int MN, int Krows, 
 // out-of-range elements read as zero.
 bool make_operand_map(CUtensorMap* map, const bf16* base, int K, int rows, int workers, long long worker_pitch = 0,
                       int box_rows = BM) {
-    EncodeTiledFn fn = encode_fn();
+    EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     if (!worker_pitch) worker_pitch = (long long)K * rows;  // dense blocks unless the operand lives inside a wider row
     cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)workers};
@@ -687,40 +635,27 @@ bool balloc(BF16State* st, T** p, size_t n) {
 }
 
 // Tile width for an output with N columns: 256 halves the operand re-reads out of L2 per output byte.
-// The wide tile only when it still leaves at least one tile per SM (148 on B200; small problems keep
-// more CTAs busy with 128-wide tiles).
-int tile_bn(int N, int M, int workers) {
+// The wide tile only when it still leaves at least one tile per SM (small problems keep more CTAs busy
+// with 128-wide tiles).
+int tile_bn(int N, int M, int workers, int sm_count) {
     if (N < 256) return 128;
     const long long wide_tiles = (long long)((N + 255) / 256) * ((M + BM - 1) / BM) * workers;
-    return wide_tiles >= 148 ? 256 : 128;
-}
-
-// multiprocessor count and shared-memory opt-in are per device: looked up for the current device
-int current_device_sms(int* dev_out) {
-    static int sms[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    if (!sms[dev]) cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
-    *dev_out = dev;
-    return sms[dev];
+    return wide_tiles >= sm_count ? 256 : 128;
 }
 
 template <bool AMN, bool BMN>
-int run_tc_major(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
-    const int bn = tile_bn(g.N, g.M, workers);
+int run_tc_major(const dbw_handle* h, const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s) {
+    const int bn = tile_bn(g.N, g.M, workers, h->sm_count);
     const int tiles_n = (g.N + bn - 1) / bn, tiles_m = (g.M + BM - 1) / BM;
     const int n_tiles = tiles_n * tiles_m * workers;
-    int dev = 0;
-    const int sms = current_device_sms(&dev);
-    if (sms <= 0) return DBW_ERR_CUDA;
-    const int grid = n_tiles < sms ? n_tiles : sms;
-    static bool configured_dev[64] = {};
-    bool& configured = configured_dev[dev];
-    if (!configured) {
+    const int grid = n_tiles < h->sm_count ? n_tiles : h->sm_count;
+    static PerDeviceOnce once;
+    const int rc = once.run(h->device, []() -> int {
         DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<4, 128, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(4, 128)));
         DBW_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<3, 256, 2, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(3, 256)));
-        configured = true;
-    }
+        return DBW_OK;
+    });
+    if (rc) return rc;
     if (bn == 128)
         gemm_tc_kernel<4, 128, 2, AMN, BMN><<<grid, GEMM_THREADS, gemm_smem(4, 128), s>>>(a, b, g, tiles_m, tiles_n, n_tiles);
     else
@@ -729,11 +664,11 @@ int run_tc_major(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, in
     return DBW_OK;
 }
 
-int run_tc(const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s, bool a_mn = false,
-           bool b_mn = false) {
-    if (a_mn && b_mn) return run_tc_major<true, true>(a, b, g, workers, s);
-    if (b_mn) return run_tc_major<false, true>(a, b, g, workers, s);
-    return run_tc_major<false, false>(a, b, g, workers, s);
+int run_tc(const dbw_handle* h, const CUtensorMap& a, const CUtensorMap& b, const TcArgs& g, int workers, cudaStream_t s,
+           bool a_mn = false, bool b_mn = false) {
+    if (a_mn && b_mn) return run_tc_major<true, true>(h, a, b, g, workers, s);
+    if (b_mn) return run_tc_major<false, true>(h, a, b, g, workers, s);
+    return run_tc_major<false, false>(h, a, b, g, workers, s);
 }
 }  // namespace
 
@@ -753,11 +688,7 @@ int grad_bf16_alloc(dbw_handle* h) {
     const size_t NB = (size_t)N * B;
     for (int l = 0; l < L && ok; ++l) {
         ok = ok && balloc(st, &st->A[l], NB * m.dims[l]);
-        if (l <= L - 2) {
-        }
-        if (l >= 1) {
-            ok = ok && balloc(st, &st->dZ[l], NB * m.dims[l]);
-        }
+        if (l >= 1) ok = ok && balloc(st, &st->dZ[l], NB * m.dims[l]);
     }
     bf16* shadow = nullptr;
     ok = ok && balloc(st, &shadow, (size_t)N * h->ld);
@@ -768,7 +699,7 @@ int grad_bf16_alloc(dbw_handle* h) {
     if (!ok) return DBW_ERR_CUDA;
     for (int l = 0; l <= L - 2; ++l) {
         ok = ok && make_operand_map(&st->fwdA[l], st->A[l], m.dims[l], B, N);
-        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1], B, N));
+        ok = ok && make_operand_map(&st->fwdB[l], st->Wh[l], m.dims[l], m.dims[l + 1], N, h->ld, tile_bn(m.dims[l + 1], B, N, h->sm_count));
         ok = ok && make_operand_map_mn(&st->dwA[l], st->dZ[l + 1], m.dims[l + 1], B, N);
         ok = ok && make_operand_map_mn(&st->dwB[l], st->A[l], m.dims[l], B, N);
         if (l >= 1) {
@@ -810,7 +741,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         B, m.dims[0], h->feat, (long long)h->S * m.dims[0], m.dims[0], batch_idx, B, h->S, st->A[0], (long long)B * m.dims[0],
         h->d_status);
     DBW_LAUNCHED();
-    gather_labels_kernel<<<N, 128, 0, s>>>(B, h->S, h->labels, batch_idx, st->ylab);
+    gather_labels_kernel<<<N, 128, 0, s>>>(B, h->S, C, h->labels, batch_idx, st->ylab, h->d_status);
     DBW_LAUNCHED();
     // forward through the tensor-core layers
     for (int l = 0; l <= L - 2; ++l) {
@@ -819,7 +750,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.out = st->A[l + 1]; g.out_z = (long long)B * g.N; g.out_pitch = g.N;
         g.bias = X + m.b_off[l]; g.bias_z = h->ld;
         g.status = h->d_status;
-        if ((rc = run_tc(st->fwdA[l], st->fwdB[l], g, N, s))) return rc;
+        if ((rc = run_tc(h, st->fwdA[l], st->fwdB[l], g, N, s))) return rc;
     }
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
@@ -856,7 +787,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         w.M = out; w.N = in; w.K = B; w.epi = EPI_DW;
         w.outf = G + m.w_off[l]; w.outf_z = h->ld; w.outf_pitch = in;
         w.status = h->d_status;
-        if ((rc = run_tc(st->dwA[l], st->dwB[l], w, N, s, true, true))) return rc;
+        if ((rc = run_tc(h, st->dwA[l], st->dwB[l], w, N, s, true, true))) return rc;
         bias_grad_bf16_kernel<<<dim3((out + 127) / 128, N), 256, 0, s>>>(out, B, st->dZ[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
         DBW_LAUNCHED();
         if (l >= 1) {
@@ -865,7 +796,7 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
             a.out = st->dZ[l]; a.out_z = (long long)B * in; a.out_pitch = in;
             a.mask = st->A[l]; a.mask_z = (long long)B * in; a.mask_pitch = in;
             a.status = h->d_status;
-            if ((rc = run_tc(st->daA[l], st->daB[l], a, N, s, false, true))) return rc;
+            if ((rc = run_tc(h, st->daA[l], st->daB[l], a, N, s, false, true))) return rc;
         }
     }
     return DBW_OK;

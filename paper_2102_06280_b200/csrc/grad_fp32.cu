@@ -8,7 +8,8 @@ namespace dbw {
 namespace {
 
 // ------------------------------------------------------------------ batch gather
-__global__ void gather_batch_kernel(int B, int S, int in_dim, const float* __restrict__ feat,
+// A sample index outside [0, S) or a label outside [0, C) is clamped and reported in the status word.
+__global__ void gather_batch_kernel(int B, int S, int in_dim, int C, const float* __restrict__ feat,
                                     const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
                                     float* __restrict__ A0, int32_t* __restrict__ ylab, uint32_t* status) {
     const int s = blockIdx.x, i = blockIdx.y;
@@ -25,7 +26,14 @@ __global__ void gather_batch_kernel(int B, int S, int in_dim, const float* __res
     } else {
         for (int k = threadIdx.x; k < in_dim; k += blockDim.x) to[k] = from[k];
     }
-    if (threadIdx.x == 0) ylab[(size_t)i * B + s] = labels[(size_t)i * S + src];
+    if (threadIdx.x == 0) {
+        int y = labels[(size_t)i * S + src];
+        if (y < 0 || y >= C) {
+            atomicOr(status, DBW_STATUS_BAD_INDEX);
+            y = y < 0 ? 0 : C - 1;
+        }
+        ylab[(size_t)i * B + s] = y;
+    }
 }
 
 // ------------------------------------------------------------------ batched strided GEMM
@@ -230,7 +238,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
                      cudaStream_t s) {
     const dbw_model_desc& m = h->model;
     const int B = m.batch, L = m.n_layers, N = h->N;
-    gather_batch_kernel<<<dim3(B, N), 128, 0, s>>>(B, h->S, m.dims[0], h->feat, h->labels, batch_idx,
+    gather_batch_kernel<<<dim3(B, N), 128, 0, s>>>(B, h->S, m.dims[0], m.dims[L], h->feat, h->labels, batch_idx,
                                                    h->d_act[0], h->d_ylab, h->d_status);
     DBW_LAUNCHED();
     int rc;

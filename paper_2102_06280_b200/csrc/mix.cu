@@ -6,6 +6,8 @@
 // of shared-memory rows, written once with 128-bit stores.  Each element of X and G is read from
 // HBM once and each element of X' is written once (12 bytes per parameter element).  A panel is
 // fully staged before any of it is written and panels are disjoint, so X' may overwrite X.
+// G == nullptr in any of the kernels means G = 0 (a consensus-only round): nothing of G is read, 8 bytes
+// per element.
 #include "common.cuh"
 
 namespace dbw {
@@ -46,7 +48,7 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             if (c < ld) {
                 v = ldg4(X + (size_t)r * ld + c);
-                if (!mix_then_correct) {
+                if (G && !mix_then_correct) {
                     const float4 g = ldg4(G + (size_t)r * ld + c);
                     const float nlr = -(lr_pw ? lr_pw[r] : lr);
                     v = fma4(nlr, g, v);
@@ -73,7 +75,7 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
                 acc = fma4(w.w, sm[j.w * GS + q], acc);
             }
             if (c < ld) {
-                if (mix_then_correct) {
+                if (G && mix_then_correct) {
                     const float4 g = ldg4(G + (size_t)i * ld + c);
                     acc = fma4(-(lr_pw ? lr_pw[i] : lr), g, acc);
                 }
@@ -101,7 +103,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
         if (c >= ld) continue;
         auto stepped = [&](int r) {
             float4 v = ldg4(X + (size_t)r * ld + c);
-            if (!mix_then_correct) v = fma4(-(lr_pw ? lr_pw[r] : lr), ldg4(G + (size_t)r * ld + c), v);
+            if (G && !mix_then_correct) v = fma4(-(lr_pw ? lr_pw[r] : lr), ldg4(G + (size_t)r * ld + c), v);
             return v;
         };
         const float ws = plan.w_self[i];
@@ -119,7 +121,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
             acc = fma4(pw[k + 3], v3, acc);
         }
         for (; k < cnt; ++k) acc = fma4(pw[k], stepped(pi[k]), acc);
-        if (mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
+        if (G && mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
         *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
         if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
     }
@@ -143,12 +145,12 @@ template <int GS>
 int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                  uint16_t* shadow, cudaStream_t s) {
     const size_t smem = (size_t)h->N * GS * 16;
-    static bool configured[64] = {};
-    if (!configured[h->device & 63]) {
-        DBW_CUDA(cudaFuncSetAttribute(mix_panel_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      h->smem_optin));
-        configured[h->device & 63] = true;
-    }
+    static PerDeviceOnce once;
+    const int rc = once.run(h->device, [h]() -> int {
+        DBW_CUDA(cudaFuncSetAttribute(mix_panel_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin));
+        return DBW_OK;
+    });
+    if (rc) return rc;
     int per_sm = 0;
     DBW_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mix_panel_kernel<GS>, kMixThreads, smem));
     if (per_sm < 1) return DBW_ERR_BAD_SHAPE;

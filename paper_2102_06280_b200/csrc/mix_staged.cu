@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
                 const bool ok = c_ok && r < N;
                 x[u] = ok ? ldg4(a.X + (size_t)r * a.ld + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            if (!a.mix_then_correct) {
+            if (a.G && !a.mix_then_correct) {  // G == nullptr: consensus-only round, G = 0
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int r = (bt + u) * 32 + p_row;
@@ -232,7 +232,7 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
                 acc.x *= w; acc.y *= w; acc.z *= w; acc.w *= w;
             }
             if (c < a.ld) {
-                if (a.mix_then_correct) {
+                if (a.G && a.mix_then_correct) {
                     const float4 gi = ldg4(a.G + (size_t)i * a.ld + c);
                     const float nlr = -(a.lr_pw ? a.lr_pw[i] : a.lr);
                     acc.x = fmaf(nlr, gi.x, acc.x); acc.y = fmaf(nlr, gi.y, acc.y);
@@ -308,12 +308,13 @@ int launch_mix_staged(dbw_handle* h, const float* X, const float* G, float lr, c
     a.plan_row = (h->maxdeg + 7) / 8 * 8;
     a.X = X; a.G = G; a.lr = lr; a.lr_pw = lr_pw; a.Xout = X_out; a.shadow = shadow; a.plan = h->plan;
     const size_t smem = staged_smem(h, a.plan_row);
-    static bool configured[64] = {};
-    if (!configured[h->device & 63]) {
+    static PerDeviceOnce once;
+    const int rc = once.run(h->device, [h]() -> int {
         DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
         DBW_CUDA(cudaFuncSetAttribute(mix_staged_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 256));
-        configured[h->device & 63] = true;
-    }
+        return DBW_OK;
+    });
+    if (rc) return rc;
     const int grid = a.n_panels < h->sm_count ? a.n_panels : h->sm_count;
     if (h->flags & DBW_WEIGHT_UNIFORM)
         mix_staged_kernel<false><<<grid, kThreads, smem, s>>>(a);

@@ -29,13 +29,13 @@
 //   warps 6-21  producers: x and g (each CTA its own 128 columns: 512-byte row segments), x~ and its
 //               three pieces, stored as MN-major 128-byte-swizzled BF16 tiles, 4-stage ring of 32 inputs
 // HBM traffic is the algorithmic 12 bytes per element; S (2 MB) is re-read from L2 for every item.
-// Every mbarrier wait is bounded; a wait that runs out sets DBW_STATUS_WAIT_TIMEOUT and goes on, so
-// all roles reach the end and tensor memory is released.
-#include <cuda.h>
-
+// Every mbarrier wait is bounded; the first wait that runs out sets DBW_STATUS_WAIT_TIMEOUT and the abort
+// word of both CTAs, after which every role stops issuing work and reaches the end, where tensor memory
+// is released.
 #include <new>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace dbw {
 
@@ -63,7 +63,8 @@ constexpr int kPrefetchAhead = 4;  // K chunks of X and G requested into L2 ahea
 // kind::f16: D = f32, A = B = bf16, A K-major, B MN-major, N = 256, M = 256 (two CTAs)
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kPanel >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using namespace ptx;
+
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -79,45 +80,33 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// arrive on a barrier given by its shared::cluster address (own CTA's or the peer's)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return;
-    atomicOr(status, DBW_STATUS_WAIT_TIMEOUT);
-}
+// Every wait is bounded and shares the CTA's abort word (set by the first wait that runs out, in both
+// CTAs of the pair): after one expired wait all roles of the pair drain at once.
 // Waits that are not on the MMA thread's critical path poll with a pause in between: a tight poll
 // loop floods the memory-instruction queue its scheduler shares with the warps that do the work.
-__device__ __forceinline__ void mbar_wait_paused(uint64_t* bar, uint32_t parity, uint32_t* status, unsigned pause_ns) {
-    for (uint32_t i = 0; i < kSpinLimit / 4; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
-        __nanosleep(pause_ns);
-    }
-    atomicOr(status, DBW_STATUS_WAIT_TIMEOUT);
+struct WaitCtx {
+    volatile uint32_t* abort;  // this CTA's abort word (shared memory)
+    uint32_t peer_abort;       // shared::cluster address of the other CTA's abort word
+    uint32_t* status;
+};
+__device__ __forceinline__ void raise_peer(const WaitCtx& w) {
+    asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(w.peer_abort), "r"(1u) : "memory");
 }
-// One lane polls for the whole warp.
-__device__ __forceinline__ void mbar_wait_warp(uint64_t* bar, uint32_t parity, uint32_t* status, unsigned pause_ns) {
-    if ((threadIdx.x & 31) == 0) mbar_wait_paused(bar, parity, status, pause_ns);
-    __syncwarp();
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
+    if (mbar_wait_bounded<true>(bar, parity, kSpinLimit, 0, w.abort, w.status)) return true;
+    raise_peer(w);
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait_paused(uint64_t* bar, uint32_t parity, const WaitCtx& w, unsigned pause_ns) {
+    if (mbar_wait_bounded<true>(bar, parity, kSpinLimit / 4, pause_ns, w.abort, w.status)) return true;
+    raise_peer(w);
+    return false;
+}
+// One lane polls for the whole warp; the result is warp-uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, const WaitCtx& w, unsigned pause_ns) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait_paused(bar, parity, w, pause_ns);
+    return __all_sync(0xffffffffu, ok);
 }
 // 2-D tiled TMA load into this CTA's shared memory; the bytes are counted on the barrier at
 // `bar_cluster_addr`, which may belong to the other CTA of the pair (no multicast).
@@ -131,8 +120,6 @@ __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* m
 __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
     asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
 }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // arrives on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far are complete
 __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -146,42 +133,8 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// K-major tile staged by TMA with the 128-byte swizzle: rows 128 bytes (64 bf16) apart, groups of
-// 8 rows 1024 bytes apart (stride byte offset); descriptor version 1, layout type 2 (128-byte swizzle).
-__device__ __forceinline__ uint64_t kmajor_sw128_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-// MN-major tile in chunks of 64 columns x 32 K rows: a K row is 128 bytes, groups of 8 K rows are
-// 1024 bytes apart (stride byte offset), the next 64 columns follow 4096 bytes on (leading byte offset).
-__device__ __forceinline__ uint64_t mnmajor_sw128_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((kKB * 128) >> 4) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
+// MN-major piece tiles of this file: chunks of 64 columns x kKB K rows
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t smem_addr) { return mnmajor_sw128_desc(smem_addr, kKB * 128); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     uint32_t r;
@@ -208,7 +161,9 @@ struct Barriers {
     uint64_t a_full[kAStages], a_empty[kAStages];
     uint64_t b_full[kBStages], b_empty[kBStages];
     uint64_t acc_full[kTiles], acc_empty[kTiles];
+    uint64_t drain;  // shutdown after an expired wait: completion of the MMAs issued so far
     uint32_t tmem_slot;
+    uint32_t abort;  // set (in both CTAs) by the first wait that runs out
 };
 
 // A work item is (panel of 256 columns, group of 512 output workers).  With more than 512 workers
@@ -234,6 +189,8 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
     const int n_tiles = min(kTiles, (a.N - row_base + 255) / 256);
 
     if (tid == 0) {
+        bars->abort = 0u;
+        mbar_init(&bars->drain, 1);
         for (int s = 0; s < kAStages; ++s) {
             mbar_init(&bars->a_full[s], 1);   // the leader's expect_tx arrival; TMA bytes of both CTAs
             mbar_init(&bars->a_empty[s], 1);  // one commit
@@ -257,6 +214,7 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
+    const WaitCtx wc{&bars->abort, map_to_cta(smem_u32(&bars->abort), rank ^ 1u), a.status};
 
     // All pairs would otherwise reach their epilogues at the same moment and the whole GPU would store
     // in bursts: start the groups of pairs spread over about one work item's time.
@@ -275,46 +233,64 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
                 const long long col = (long long)(group + w * groups) * kPanel + (long long)rank * kHalf;
                 if (col >= a.ld) return;
                 tma_prefetch_2d(&tmX, (int)col, kc * kKC);
-                if (!a.mix_then_correct) tma_prefetch_2d(&tmG, (int)col, kc * kKC);
+                if (a.G && !a.mix_then_correct) tma_prefetch_2d(&tmG, (int)col, kc * kKC);
             };
             for (int ch = 0; ch < kPrefetchAhead; ++ch) prefetch(ch);
             int it = 0;
-            for (int w = 0; w < my_items; ++w)
+            bool live = true;
+            for (int w = 0; w < my_items && live; ++w)
                 for (int kc = 0; kc < a.n_kc; ++kc, ++it) {
                     prefetch(it + kPrefetchAhead);
                     const int s = it % kAStages;
-                    if (it >= kAStages) mbar_wait_paused(&bars->a_empty[s], ((it / kAStages) - 1) & 1, a.status, 64);
+                    if (it >= kAStages && !mbar_wait_paused(&bars->a_empty[s], ((it / kAStages) - 1) & 1, wc, 64)) {
+                        live = false;  // a wait ran out somewhere in the pair: issue nothing more
+                        break;
+                    }
                     if (rank == 0) mbar_expect_tx(&bars->a_full[s], (uint32_t)(2 * n_tiles * kTileBytes));
                     const uint32_t full_addr = map_to_cta(smem_u32(&bars->a_full[s]), 0);
                     for (int t = 0; t < n_tiles; ++t)
                         tma_load_2d_pair(ringA + s * kAStageBytes + t * kTileBytes, &tmS, kc * kKC, row_base + t * 256 + (int)rank * 128,
                                          full_addr);
                 }
+            // The copies of both CTAs are counted on the leader's barriers: the leader sees the last ones land
+            // before the pair meets at the final cluster barrier, so neither CTA leaves with a copy in flight.
+            if (rank == 0)
+                for (int j = it > kAStages ? it - kAStages : 0; j < it; ++j) mbar_wait_quiet<true>(&bars->a_full[j % kAStages], (j / kAStages) & 1, 1u << 20);
         }
     } else if (warp == 1) {
         // ---------------- MMA issue (leader CTA only) ----------------
         if (rank == 0 && lane == 0) {
             int it = 0;
-            for (int w = 0; w < my_items; ++w)
-                for (int kc = 0; kc < a.n_kc; ++kc, ++it) {
+            bool live = true;
+            for (int w = 0; w < my_items && live; ++w)
+                for (int kc = 0; kc < a.n_kc && live; ++kc, ++it) {
                     const int sa = it % kAStages;
-                    mbar_wait(&bars->a_full[sa], (it / kAStages) & 1, a.status);
+                    if (!mbar_wait(&bars->a_full[sa], (it / kAStages) & 1, wc)) {
+                        live = false;
+                        break;
+                    }
                     const uint32_t baseA = smem_u32(ringA + sa * kAStageBytes);
 #pragma unroll
                     for (int hb = 0; hb < kKC / kKB; ++hb) {  // the two halves of the K chunk: one piece-ring stage each
                         const int ib = it * (kKC / kKB) + hb, sb = ib % kBStages;
-                        mbar_wait(&bars->b_full[sb], (ib / kBStages) & 1, a.status);
+                        if (!mbar_wait(&bars->b_full[sb], (ib / kBStages) & 1, wc)) {
+                            live = false;
+                            break;
+                        }
                         tc_fence_after();
                         const uint32_t baseB = smem_u32(ringB + sb * kBStageBytes);
                         for (int t = 0; t < n_tiles; ++t) {
                             if (kc == 0 && hb == 0 && w > 0) {  // the epilogues of both CTAs have drained this tile's accumulator
-                                mbar_wait(&bars->acc_empty[t], (w - 1) & 1, a.status);
+                                if (!mbar_wait(&bars->acc_empty[t], (w - 1) & 1, wc)) {
+                                    live = false;
+                                    break;
+                                }
                                 tc_fence_after();
                             }
                             const uint64_t da = kmajor_sw128_desc(baseA + t * kTileBytes) + (uint64_t)(hb * (kKB / 16) * 2);
 #pragma unroll
                             for (int pc = 0; pc < 3; ++pc) {
-                                const uint64_t db = mnmajor_sw128_desc(baseB + pc * kPieceBytes);
+                                const uint64_t db = mnmajor_desc(baseB + pc * kPieceBytes);
 #pragma unroll
                                 for (int k = 0; k < kKB / 16; ++k)  // 16 inputs further: 32 bytes (K-major), 16 rows of 128 bytes (MN-major)
                                     tc_mma_pair(tmem_base + (uint32_t)(t * kPanel), da + (uint64_t)(k * 2), db + (uint64_t)(k * 128),
@@ -322,10 +298,15 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
                             }
                             if (kc == a.n_kc - 1 && hb == kKC / kKB - 1) tc_commit_pair(&bars->acc_full[t]);
                         }
+                        if (!live) break;
                         tc_commit_pair(&bars->b_empty[sb]);
                     }
-                    tc_commit_pair(&bars->a_empty[sa]);
+                    if (live) tc_commit_pair(&bars->a_empty[sa]);
                 }
+            if (bars->abort) {  // shutdown after an expired wait: the MMAs issued so far are complete before tensor memory is freed
+                tc_commit_pair(&bars->drain);
+                mbar_wait_quiet<true>(&bars->drain, 0, 1u << 20);
+            }
         }
     } else if (warp < 2 + kEpiWarps) {
         // ---------------- epilogue: this warp owns accumulator lanes 32 q .. 32 q + 31 ----------------
@@ -348,7 +329,7 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
 #pragma unroll
             for (int t = 0; t < kTiles; ++t) {
                 if (t >= n_tiles) break;
-                mbar_wait_warp(&bars->acc_full[t], w & 1, a.status, 256);
+                if (!mbar_wait_warp(&bars->acc_full[t], w & 1, wc, 256)) break;
                 tc_fence_after();
                 const int row0 = row_base + t * 256 + (int)rank * 128 + q * 32;
                 for (int c = 0; c < kPanel / 32; ++c, ++blk) {
@@ -385,7 +366,7 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
                             const int gi = row0 + rr;
                             float4 v = *reinterpret_cast<const float4*>(buf + rr * 128 + ((f4 ^ (rr & 7)) << 4));
                             if (gi < a.N && col < a.ld) {
-                                if (a.mix_then_correct) {
+                                if (a.mix_then_correct && a.G) {
                                     const float4 g = __ldg(reinterpret_cast<const float4*>(a.G + (size_t)gi * a.ld + col));
                                     const float nlr = -(a.lr_pw ? a.lr_pw[gi] : a.lr);
                                     v.x = fmaf(nlr, g.x, v.x); v.y = fmaf(nlr, g.y, v.y);
@@ -429,10 +410,10 @@ mix_tc_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
                 const int row = row_lo + j0 + 4 * (q & 1) + 16 * (q >> 1);
                 const bool ok = row < a.N && col < a.ld;
                 x[q] = ok ? __ldg(reinterpret_cast<const float4*>(a.X + (size_t)row * a.ld + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                g[q] = (ok && !a.mix_then_correct) ? __ldg(reinterpret_cast<const float4*>(a.G + (size_t)row * a.ld + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                g[q] = (ok && a.G && !a.mix_then_correct) ? __ldg(reinterpret_cast<const float4*>(a.G + (size_t)row * a.ld + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             const int sb = hc % kBStages;
-            if (hc >= kBStages) mbar_wait_warp(&bars->b_empty[sb], ((hc / kBStages) - 1) & 1, a.status, 64);
+            if (hc >= kBStages && !mbar_wait_warp(&bars->b_empty[sb], ((hc / kBStages) - 1) & 1, wc, 64)) break;
             uint8_t* stage = ringB + sb * kBStageBytes;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -483,22 +464,6 @@ build_selection_kernel(int N, int k_pad, MixPlan plan, uint16_t* S) {
     const int cnt = plan.cnt[i];
     for (int k = threadIdx.x; k < cnt; k += blockDim.x) S[(size_t)i * k_pad + plan.idx[(size_t)i * plan.stride + k]] = 0x3F80u;
     if (threadIdx.x == 0) S[(size_t)i * k_pad + i] = 0x3F80u;
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
 }
 
 // launch configuration of `ctas` CTAs in clusters of two
@@ -556,7 +521,7 @@ static int mix_tc_prepare(dbw_handle* h) {
     st->rows_pad = (h->N + 255) / 256 * 256;
     st->k_pad = (h->N + kKC - 1) / kKC * kKC;
     DBW_CUDA(cudaMalloc(reinterpret_cast<void**>(&st->S), (size_t)st->rows_pad * st->k_pad * 2));
-    EncodeTiledFn fn = encode_fn();
+    EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return DBW_ERR_CUDA;
     cuuint64_t dims[2] = {(cuuint64_t)st->k_pad, (cuuint64_t)st->rows_pad};
     cuuint64_t strides[1] = {(cuuint64_t)st->k_pad * 2};
@@ -584,7 +549,7 @@ int launch_mix_tc(dbw_handle* h, const float* X, const float* G, float lr, const
     TcMixState* st = h->mix_tc;
     // tensor maps of X' (the epilogue's stores) and of X and G (L2 prefetch), [N][ld] fp32; rebuilt when a pointer changes
     auto encode = [&](CUtensorMap* map, const float* base, cuuint32_t box_cols, cuuint32_t box_rows, CUtensorMapSwizzle sw) {
-        EncodeTiledFn fn = encode_fn();
+        EncodeTiledFn fn = encode_tiled_fn();
         cuuint64_t dims[2] = {(cuuint64_t)h->ld, (cuuint64_t)h->N};
         cuuint64_t strides[1] = {(cuuint64_t)h->ld * 4};
         cuuint32_t box[2] = {box_cols, box_rows};
@@ -600,7 +565,7 @@ int launch_mix_tc(dbw_handle* h, const float* X, const float* G, float lr, const
         if (!encode(&st->x_map, X, kHalf, kKC, CU_TENSOR_MAP_SWIZZLE_NONE)) return DBW_ERR_CUDA;
         st->x_ptr = X;
     }
-    if (st->g_ptr != G) {
+    if (G && st->g_ptr != G) {  // G == nullptr (consensus only): the kernel never touches the map
         if (!encode(&st->g_map, G, kHalf, kKC, CU_TENSOR_MAP_SWIZZLE_NONE)) return DBW_ERR_CUDA;
         st->g_ptr = G;
     }

@@ -162,7 +162,10 @@ select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restri
     }
 }
 
-// Plan from a caller-supplied kept mask (dbw_mix on its own).
+// Plan from a caller-supplied kept mask (dbw_mix on its own).  With uniform weights the weight is
+// 1 / (1 + number of kept entries in the mask), so a row's weights sum to one whatever the mask holds;
+// a mask whose count differs from deg_i - b_i is reported (DBW_STATUS_BAD_B).  The weights of Assumption 1
+// use the nominal counts p = deg - b of both ends and keep the rows stochastic through w_ii = 1 - sum.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 plan_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
             const uint8_t* __restrict__ kept, const int32_t* __restrict__ b, uint32_t* status, MixPlan plan,
@@ -171,7 +174,14 @@ plan_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restrict
     const int i = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (i >= N) return;
     const int lo = rowptr[i], hi = rowptr[i + 1], deg = hi - lo;
-    const int p = deg - clamped_b(b, i, deg, status);
+    int p = deg - clamped_b(b, i, deg, status);
+    int n_kept = 0;
+    for (int base = 0; base < deg; base += 32) {
+        const int e = lo + base + lane;
+        n_kept += __popc(__ballot_sync(0xffffffffu, e < hi && kept[e] != 0));
+    }
+    if (n_kept != p && lane == 0) atomicOr(status, DBW_STATUS_BAD_B);
+    if (uniform) p = n_kept;
     float wsum = 0.f;
     int running = 0;
     for (int base = 0; base < deg; base += 32) {
@@ -226,17 +236,19 @@ constexpr size_t kStaticBytes = kStaticTnbrOff + sizeof(double) * DBW_SELECT_STA
 static __device__ __align__(256) unsigned char g_select_scratch[kStaticBytes];
 
 // Device address of the scratch on the current device (the symbol's name is only a host-side
-// stand-in); looked up once per device.
+// stand-in); looked up once per device, under a lock, so host threads may race for the first call.
 int static_scratch(unsigned char** out) {
+    static PerDeviceOnce once;
     static unsigned char* cache[64] = {};
     int dev = 0;
     DBW_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return DBW_ERR_BAD_SHAPE;
-    if (!cache[dev]) {
+    const int rc = once.run(dev, [dev]() -> int {
         void* p = nullptr;
         DBW_CUDA(cudaGetSymbolAddress(&p, g_select_scratch));
         cache[dev] = static_cast<unsigned char*>(p);
-    }
+        return DBW_OK;
+    });
+    if (rc) return rc;
     *out = cache[dev];
     return DBW_OK;
 }

@@ -7,11 +7,14 @@ For them the library carries a fixed scratch array and a handle-free entry point
 calls it through the C ABI twice in a row (the second call finds the first call's leftovers in
 the shared scratch) and requires the same bytes as the handle-based dbw_select, which runs the
 same kernel: kept masks and all times are compared bit for bit, as everywhere in these tests.
+Since that compares the CUDA path with itself, the outputs are also compared, bit for bit, with the
+CPU oracle's selection and times (Section 2.2, Section 3.2.2).
 The file name sorts last so that a `-x` run has already executed every other test.
 """
 import numpy as np
 import pytest
 
+from oracle import dbw_oracle as orc
 from workloads import configs as wl
 
 pytestmark = pytest.mark.gpu
@@ -51,6 +54,11 @@ def test_static_selection_matches_handle_based_selection_twice():
             for a, r in zip(got, ref):
                 assert torch.equal(a, r)
             assert int(st.item()) == 0
+            o_kept = orc.select_fastest(rowptr, col, t, b)
+            o_Tn, o_Tw, o_Tr = orc.round_times(rowptr, col, t, b, o_kept)
+            assert np.array_equal(got[0].cpu().numpy(), o_kept)
+            assert np.array_equal(got[1].cpu().numpy(), o_Tw) and np.array_equal(got[2].cpu().numpy(), o_Tn)
+            assert float(got[3].cpu()[0]) == o_Tr
         # device-detected problems are reported through status_out, results stay clamped
         bad = dev(np.full(n, -3, dtype=np.int32))
         binding.select_static(rp_d, col_d, t_d, bad, *got, status_out=st)
