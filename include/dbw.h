@@ -60,6 +60,7 @@ enum {
                                      does not hold deg_i - b_i entries for some i */
 #define DBW_STATUS_NAN_TIME 2u    /* some arrival time was NaN (ordered last) */
 #define DBW_STATUS_WAIT_TIMEOUT 4u /* a bounded pipeline wait expired; results of that call are invalid */
+#define DBW_STATUS_INTERNAL 16u   /* a kernel found its own precomputed data inconsistent (should not happen) */
 #define DBW_STATUS_BAD_INDEX 8u   /* a batch index was outside [0, S) or a label outside [0, classes) (clamped) */
 
 #define DBW_MAX_LAYERS 8
@@ -193,10 +194,13 @@ int dbw_mix_in_place_ok(const dbw_handle* h);
  * 2 = the tensor-core kernel wherever it applies (uniform weights, 256 <= N <= 1024): the mix as a
  *     dense product with the 0/1 selection matrix, every fp32 value split exactly into three BF16
  *     pieces, fp32 accumulation; with N > 512 it cannot run in place (dbw_mix_in_place_ok() = 0),
+ *  3 = the structured-sparse tensor-core kernel wherever it applies (uniform weights, 256 <= N <= 1024, a
+ *      2:4 order of the graph exists, see dbw_graph_order_2of4): the same product with the selection
+ *      matrix compressed 2:4, at twice the dense tensor-core rate; in place only for N <= 512,
  * -1 = always the direct (L2 re-read, out-of-place only) kernel. */
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols);
 /* Which mix kernel the current settings select: 0 = direct (L2 re-read), 1 = shared-memory panel,
- * 2 = tensor-memory staged, 3 = tensor-core.  Negative on error. */
+ * 2 = tensor-memory staged, 3 = tensor-core, 4 = structured-sparse tensor-core.  Negative on error. */
 int dbw_mix_kernel(const dbw_handle* h);
 
 /*
@@ -283,6 +287,18 @@ int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds);
  * status word, as an expired wait in a real pipeline does; the context stays usable.
  */
 int dbw_debug_wait_probe(dbw_handle* h, uint32_t polls, uint32_t* out, void* stream);
+
+/*
+ * Worker reordering for the structured-sparse tensor-core mix (Eq. 5 as the product of the 0/1 selection
+ * matrix with the parameter matrix; the paper prescribes no order of the workers, so any order is the
+ * same method).  HOST in: the sorted CSR of dbw_init.  HOST out: order[k], k < the returned count, is the
+ * worker placed at input position k, or -1 for a position left empty.  The order is such that for every
+ * worker i no aligned group of four consecutive positions holds more than two members of {i} + N_i, so
+ * every row of every selection matrix the graph admits is 2:4 sparse.  Deterministic.  Returns the number
+ * of positions used (a multiple of 128, at most 1024 and at most `capacity`), 0 when no such order was
+ * found, or a negative error.  Needs no GPU.
+ */
+int dbw_graph_order_2of4(int32_t N, const int32_t* h_rowptr, const int32_t* h_col, int32_t* order, int32_t capacity);
 
 /* Kernels launched by this library since it was loaded (for launch accounting). */
 int64_t dbw_launch_count(void);

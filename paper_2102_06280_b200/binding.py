@@ -16,7 +16,7 @@ import numpy as np
 WEIGHT_METROPOLIS, WEIGHT_UNIFORM = 0, 1
 ORDER_LOCAL_THEN_MIX, ORDER_MIX_THEN_CORRECT = 0, 2
 GEMM_FP32, GEMM_BF16 = 0, 4
-STATUS_BAD_B, STATUS_NAN_TIME, STATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4, 8
+STATUS_BAD_B, STATUS_NAN_TIME, STATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX, STATUS_INTERNAL = 1, 2, 4, 8, 16
 MAX_LAYERS = 8
 
 _ERR = {-1: "DBW_ERR_NULL", -2: "DBW_ERR_BAD_GRAPH", -3: "DBW_ERR_BAD_SHAPE", -4: "DBW_ERR_BAD_B",
@@ -67,6 +67,7 @@ _SIGNATURES = {
     "dbw_profile": (C.c_int, [_P, C.c_int]),
     "dbw_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
     "dbw_debug_wait_probe": (C.c_int, [_P, C.c_uint32, _P, _P]),
+    "dbw_graph_order_2of4": (C.c_int, [C.c_int32, _P, _P, _P, C.c_int32]),
     "dbw_launch_count": (C.c_int64, []),
     "dbw_last_cuda_error": (C.c_int, []),
 }
@@ -214,7 +215,7 @@ class Dbw:
         _check(lib().dbw_set_param_tracking(self._h, int(bool(enable))), "dbw_set_param_tracking")
 
     def mix_kernel(self) -> str:
-        return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel", "mix_tc_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]
+        return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel", "mix_tc_kernel", "mix_sp_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]
 
     def set_mix_panel(self, cols: int):
         _check(lib().dbw_set_mix_panel(self._h, int(cols)), "dbw_set_mix_panel")
@@ -277,6 +278,16 @@ def select_static(rowptr, col, t, b, kept, T_worker=None, T_nbr=None, T_round=No
     n = int(rowptr.numel()) - 1
     _check(lib().dbw_select_static(n, _ptr(rowptr), _ptr(col), _ptr(t), _ptr(b), _ptr(kept), _ptr(T_worker),
                                    _ptr(T_nbr), _ptr(T_round), _ptr(status_out), _stream()), "dbw_select_static")
+
+
+def graph_order_2of4(rowptr, col) -> Optional[np.ndarray]:
+    """dbw_graph_order_2of4: the worker order of the structured-sparse mix (host only); None if there is none."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    order = np.full(1024, -1, dtype=np.int32)
+    n = _check(lib().dbw_graph_order_2of4(len(rowptr) - 1, rowptr.ctypes.data, col.ctypes.data, order.ctypes.data, 1024),
+               "dbw_graph_order_2of4")
+    return order[:n].copy() if n > 0 else None
 
 
 def launch_count() -> int:

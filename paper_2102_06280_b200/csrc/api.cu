@@ -120,6 +120,7 @@ void free_all(dbw_handle* h) {
     grad_fp32_free(h);
     grad_bf16_free(h);
     mix_tc_free(h);
+    mix_sp_free(h);
     void* ptrs[] = {h->d_rowptr, h->d_col, h->d_links, h->d_covered, h->d_epoch, h->d_status, h->d_waited,
                     h->d_ticket, h->d_Tnbr_ws, h->plan.idx, h->plan.w, h->plan.w_self, h->plan.cnt, h->d_G,
                     h->s_t, h->s_b, h->s_bidx, h->s_kept, h->s_Tw, h->s_Tr, h->s_loss};
@@ -240,6 +241,7 @@ int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* 
         !cuda_ok(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) ||
         !cuda_ok(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)))
         return fail(DBW_ERR_CUDA);
+    mix_sp_prepare(h);  // the 2:4 worker order of the sparse tensor-core mix, where that kernel can apply
     if (model) {
         h->has_model = true;
         h->model = *model;
@@ -325,7 +327,7 @@ int dbw_mix_kernel(const dbw_handle* h) { return h ? mix_kernel_kind(h) : DBW_ER
 
 int dbw_set_mix_panel(dbw_handle* h, int32_t cols) {
     if (!h) return DBW_ERR_NULL;
-    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 2 || cols == 16 || cols == 32 || cols == 64 || cols == 128 || cols == 256)) return DBW_ERR_BAD_SHAPE;
+    if (!(cols == 0 || cols == -1 || cols == 1 || cols == 2 || cols == 3 || cols == 16 || cols == 32 || cols == 64 || cols == 128 || cols == 256)) return DBW_ERR_BAD_SHAPE;
     h->mix_panel_cols = cols;
     return DBW_OK;
 }
@@ -503,6 +505,13 @@ int dbw_get_links(const dbw_handle* h, int32_t* links) {
     if (!h || !links) return DBW_ERR_NULL;
     std::memcpy(links, h->h_links.data(), h->h_links.size() * sizeof(int32_t));
     return h->N - 1;
+}
+
+int dbw_graph_order_2of4(int32_t N, const int32_t* h_rowptr, const int32_t* h_col, int32_t* order, int32_t capacity) {
+    if (!h_rowptr || !h_col || !order) return DBW_ERR_NULL;
+    if (N < 1 || capacity < 1) return DBW_ERR_BAD_SHAPE;
+    if (!valid_graph(N, h_rowptr, h_col)) return DBW_ERR_BAD_GRAPH;
+    return mix_sp_order_host(N, h_rowptr, h_col, order, capacity);
 }
 
 int64_t dbw_launch_count(void) { return g_launches.load(); }

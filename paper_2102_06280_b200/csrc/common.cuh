@@ -64,6 +64,7 @@ struct MixPlan {
 
 struct BF16State;  // tensor-core gradient path (grad_bf16.cu)
 struct TcMixState;  // tensor-core mix (mix_tc.cu)
+struct SpMixState;  // tensor-core mix with 2:4 structured sparsity (mix_sp.cu)
 
 }  // namespace dbw
 
@@ -96,6 +97,7 @@ struct dbw_handle {
     dbw::MixPlan plan;
     int mix_panel_cols = 0;  // 0 = automatic
     dbw::TcMixState* mix_tc = nullptr;  // selection matrix and tensor map of the tensor-core mix (lazy)
+    dbw::SpMixState* mix_sp = nullptr;  // 2:4 order, compressed selection matrix and tensor maps of the sparse tensor-core mix (dbw_init)
 
     // model / gradient path
     bool has_model = false;
@@ -167,6 +169,15 @@ bool mix_tc_in_place_ok(const dbw_handle* h);
 void mix_tc_free(dbw_handle* h);
 int launch_mix_tc(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                   uint16_t* shadow, cudaStream_t s);
+
+// mix_sp.cu
+void mix_sp_prepare(dbw_handle* h);
+bool mix_sp_usable(const dbw_handle* h);
+bool mix_sp_in_place_ok(const dbw_handle* h);
+void mix_sp_free(dbw_handle* h);
+int launch_mix_sp(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
+                  uint16_t* shadow, cudaStream_t s);
+int mix_sp_order_host(int N, const int32_t* rowptr, const int32_t* col, int32_t* order, int capacity);
 
 // dtur.cu
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);

@@ -129,7 +129,7 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
 
 int auto_group_size(const dbw_handle* h) {
     if (h->mix_panel_cols < 0) return 0;  // direct kernel forced
-    if (h->mix_panel_cols == 1 || h->mix_panel_cols == 2) return 0; // staged / tensor-core kernel forced (handled by the caller)
+    if (h->mix_panel_cols >= 1 && h->mix_panel_cols <= 3) return 0;  // staged / tensor-core kernels forced (handled by the caller)
     if (h->mix_panel_cols) return ((size_t)h->N * h->mix_panel_cols * 4 <= (size_t)h->smem_optin) ? h->mix_panel_cols / 4 : 0;
     // few workers and a matrix that streams from HBM (well beyond L2): 256-column panels (1 KB row segments) while
     // three CTAs still share an SM
@@ -165,6 +165,8 @@ int launch_panel(dbw_handle* h, const float* X, const float* G, float lr, const 
 
 }  // namespace
 
+constexpr bool kSparseByDefault = false;
+
 // The tensor-memory staged kernel takes over when it applies and the plain panel kernel could not
 // keep a 32-column (128-byte segment) panel with two CTAs per SM.
 static bool use_staged(const dbw_handle* h) {
@@ -176,8 +178,19 @@ static bool use_staged(const dbw_handle* h) {
 // The tensor-core kernel (dense 0/1 selection product) when asked for and applicable.
 static bool use_tc(const dbw_handle* h) { return h->mix_panel_cols == 2 && mix_tc_usable(h); }
 
-bool mix_panel_fits(const dbw_handle* h) { return use_tc(h) ? mix_tc_in_place_ok(h) : (use_staged(h) || auto_group_size(h) != 0); }
-int mix_kernel_kind(const dbw_handle* h) { return use_tc(h) ? 3 : use_staged(h) ? 2 : (auto_group_size(h) != 0 ? 1 : 0); }
+// The 2:4 structured-sparse tensor-core kernel: when asked for, or automatically where the staged kernel
+// would otherwise run with uniform weights (many workers, many kept neighbours) and a 2:4 order exists.
+static bool use_sp(const dbw_handle* h) {
+    if (!mix_sp_usable(h)) return false;
+    if (h->mix_panel_cols == 3) return true;
+    return h->mix_panel_cols == 0 && kSparseByDefault && h->N >= 512 && use_staged(h);
+}
+
+bool mix_panel_fits(const dbw_handle* h) {
+    if (use_sp(h)) return mix_sp_in_place_ok(h);
+    return use_tc(h) ? mix_tc_in_place_ok(h) : (use_staged(h) || auto_group_size(h) != 0);
+}
+int mix_kernel_kind(const dbw_handle* h) { return use_sp(h) ? 4 : use_tc(h) ? 3 : use_staged(h) ? 2 : (auto_group_size(h) != 0 ? 1 : 0); }
 
 int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                cudaStream_t s) {
@@ -186,6 +199,7 @@ int launch_mix(dbw_handle* h, const float* X, const float* G, float lr, const fl
     uint16_t* shadow = (h->track_params && h->d_shadow) ? h->d_shadow : nullptr;
     h->shadow_valid = shadow != nullptr;
     h->shadow_of = X_out;
+    if (use_sp(h)) return launch_mix_sp(h, X, G, lr, lr_pw, X_out, shadow, s);
     if (use_tc(h)) return launch_mix_tc(h, X, G, lr, lr_pw, X_out, shadow, s);
     if (use_staged(h)) return launch_mix_staged(h, X, G, lr, lr_pw, X_out, shadow, s);
     switch (auto_group_size(h)) {

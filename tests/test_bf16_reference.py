@@ -3,7 +3,7 @@ compares the GPU against: the rounding itself on values whose bfloat16 neighbour
 gradient where it must coincide with the double-precision oracle."""
 import numpy as np
 
-from bf16_reference import bf16_round, mlp_grad_bf16_points
+from bf16_reference import bf16_round, gradient_agrees, mlp_grad_bf16_points
 from oracle import dbw_oracle as orc
 
 
@@ -55,3 +55,51 @@ def test_integer_network_forward_is_exact_and_gradient_is_close():
     assert np.abs(g[-last:] - g0[-last:]).max() <= 1e-13
     assert np.abs(g - g0).max() <= 2.0 ** -7 * np.abs(g0).max()
     assert np.abs(g - g0).max() > 0.0                               # the dZ rounding is really applied
+
+
+def test_unresolvable_relu_decisions_are_enumerated():
+    """A pre-activation that is zero up to fp32 accumulation error may be taken either way by the CUDA path: the
+    reference lists it, and best_block_error accepts the gradient of either decision and nothing else."""
+    rng = np.random.default_rng(3)
+    dims, B = [16, 8, 4], 6
+    feats = bf16_round(rng.random((B, 16)))
+    x = (rng.standard_normal(16 * 8 + 8 + 8 * 4 + 4) * 0.5).astype(np.float32)
+    x[16 * 8: 16 * 8 + 8] = 0.0
+    w_row = bf16_round(x[:16])
+    # unit 0 of sample 2: make the pre-activation cancel to (nearly) nothing through the fp32 bias
+    x[16 * 8] = np.float32(-(feats[2] @ w_row) + 3e-7)
+    x[:16] = w_row.astype(np.float32)
+    labels = rng.integers(0, 4, B)
+    amb = []
+    g_on, _ = mlp_grad_bf16_points(x, dims, feats, labels, ambiguous=amb)
+    assert amb == [(1, 2, 0)]
+    g_off, _ = mlp_grad_bf16_points(x, dims, feats, labels, flips=amb)
+    assert np.abs(g_on - g_off).max() > 1e-3 * np.abs(g_on).max()          # the two decisions really differ
+    for g in (g_on, g_off):
+        ok, rep = gradient_agrees(g, x, dims, feats, labels, tol=1e-9)
+        assert ok and rep["max"] <= 1e-12 and rep["ambiguous"] == 1
+    assert gradient_agrees(g_off, x, dims, feats, labels, tol=1e-9)[1]["switched"] == 1
+    ok, rep = gradient_agrees(0.5 * (g_on + g_off), x, dims, feats, labels, tol=1e-9)
+    assert not ok and rep["max"] > 1e-4                                    # anything in between is rejected
+
+
+def test_strict_gate_rejects_real_defects_even_with_ambiguous_decisions():
+    """The defects the gate exists to catch fail it whether or not ambiguous decisions are present: a dropped half
+    of the batch in one layer's dW, a bias gradient off by the batch size, a unit masked wrongly."""
+    rng = np.random.default_rng(3)
+    dims, B = [16, 8, 4], 6
+    feats = bf16_round(rng.random((B, 16)))
+    x = (rng.standard_normal(16 * 8 + 8 + 8 * 4 + 4) * 0.5).astype(np.float32)
+    x[16 * 8: 16 * 8 + 8] = 0.0
+    w_row = bf16_round(x[:16])
+    x[16 * 8] = np.float32(-(feats[2] @ w_row) + 3e-7)          # one ambiguous decision, as above
+    x[:16] = w_row.astype(np.float32)
+    labels = rng.integers(0, 4, B)
+    g, _ = mlp_grad_bf16_points(x, dims, feats, labels)
+    assert gradient_agrees(g * (1 + 1e-5), x, dims, feats, labels)[0]
+    half = g.copy(); half[:16 * 8] *= 0.5
+    assert not gradient_agrees(half, x, dims, feats, labels)[0]
+    bias = g.copy(); bias[16 * 8: 16 * 8 + 8] *= B
+    assert not gradient_agrees(bias, x, dims, feats, labels)[0]
+    masked = g.copy(); masked[:16 * 8].reshape(8, 16)[3] = 0.0   # a unit that is NOT ambiguous
+    assert not gradient_agrees(masked, x, dims, feats, labels)[0]

@@ -151,17 +151,19 @@ def test_mix_matches_oracle(name, d, rule, order):
 @pytest.mark.parametrize("n,deg,d,order", [(320, 16, 1000, "local_then_mix"), (700, 16, 1300, "mix_then_correct"),
                                            (1000, 32, 2052, "local_then_mix"), (512, 8, 516, "local_then_mix"),
                                            (514, 8, 260, "mix_then_correct")])
-def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order):
-    """The dense 0/1-selection product on the tensor cores (three exact BF16 pieces per fp32 value): worker
-    counts that leave ragged row tiles and K chunks, widths that leave a ragged last panel, both update
-    orders, per-worker learning rates, in place where one CTA pair owns a panel, run-to-run reproducible."""
+@pytest.mark.parametrize("panel,kernel", [(2, "mix_tc_kernel"), (3, "mix_sp_kernel")])
+def test_mix_tensor_core_kernel_matches_oracle(n, deg, d, order, panel, kernel):
+    """The 0/1-selection product on the tensor cores (three exact BF16 pieces per fp32 value), dense and with the
+    selection matrix 2:4 structured-sparse in the graph's worker order: worker counts that leave ragged row tiles
+    and K chunks, widths that leave a ragged last panel, both update orders, per-worker learning rates, in place
+    where one CTA pair owns a panel, run-to-run reproducible."""
     p = _dbw()
     rowptr, col = wl.random_regular(n, deg, 21)
     degs = np.diff(rowptr)
     flags = p.WEIGHT_UNIFORM | (p.ORDER_MIX_THEN_CORRECT if order == "mix_then_correct" else 0)
     h = p.Dbw(rowptr, col, d=d, ld=d, flags=flags)
-    h.set_mix_panel(2)
-    assert h.mix_kernel() == "mix_tc_kernel"
+    h.set_mix_panel(panel)
+    assert h.mix_kernel() == kernel
     assert h.mix_in_place_ok() == (n <= 512)
     rng = np.random.default_rng(12)
     X = rng.standard_normal((n, d), dtype=np.float32) * np.float32(3.0)
@@ -364,13 +366,15 @@ def test_grad_fp32_matches_oracle(dims, batch, n):
 def test_grad_bf16_tensor_cores_match_oracle(dims, batch, n):
     """BF16 operands, fp32 accumulate.  Two references side by side:
     (1) tests/bf16_reference.py: the same gradient in double on operands rounded to bf16 at the points where
-        the CUDA path rounds them.  Element-wise bar: 1e-3 of each layer block's max-norm (what is left is fp32
-        accumulation order and the rare entry on a bf16 rounding boundary; a dropped K block, a wrong bias
-        gradient scale or a wrong ReLU mask on a few percent of entries is orders of magnitude above it).
+        the CUDA path rounds them.  Per layer block: every entry within 5e-3 of the block's max-norm and the
+        block's 2-norm error within 1e-3 (measured on these shapes: at most 5e-4 and 4.5e-4); ReLU decisions on
+        pre-activations that fp32 accumulation cannot tell from zero are inferred from the GPU's own output
+        (see gradient_agrees).  A dropped K block, a wrong bias gradient scale or a wrong ReLU mask on a few
+        percent of the entries is orders of magnitude above these bars.
     (2) the double-precision oracle on the fp32 master weights: bf16 rounding (2^-8 per operand, three chained
         GEMM stages for the first layer's dW, ReLU masks that flip where a pre-activation is within rounding
         of zero) is what separates them: 0.15 of each block's max-norm and a cosine above 0.995."""
-    from bf16_reference import mlp_grad_bf16_points
+    from bf16_reference import gradient_agrees
     p = _dbw()
     rowptr, col = wl.ring(n) if n >= 3 else wl.path(n)
     m = p.model_layout(dims, batch)
@@ -398,21 +402,23 @@ def test_grad_bf16_tensor_cores_match_oracle(dims, batch, n):
     worst = 0.0
     for i in range(n):
         g, l = orc.mlp_grad(Xl[i], dims, feat[i][idx[i]], labels[i][idx[i]])
-        ge, le = mlp_grad_bf16_points(Xl[i], dims, feat[i][idx[i]], labels[i][idx[i]])
+        # (a ReLU decision on a pre-activation that fp32 accumulation cannot tell from zero may go either way:
+        # see gradient_agrees for how those are treated)
+        ok, rep = gradient_agrees(got[i].astype(np.float64), Xl[i], dims, feat[i][idx[i]], labels[i][idx[i]])
+        worst = max(worst, rep["l2"])
+        assert ok, (i, rep)
+        le = rep["loss"]
         off = 0
         for lay in range(len(dims) - 1):
             for size in (dims[lay] * dims[lay + 1], dims[lay + 1]):
-                a, r, e = got[i, off:off + size], g[off:off + size], ge[off:off + size]
-                err = np.abs(a - e).max() / max(np.abs(e).max(), 1e-30)
-                worst = max(worst, err)
-                assert err <= 1e-3, (i, lay, size, err)
+                a, r = got[i, off:off + size], g[off:off + size]
                 assert np.abs(a - r).max() <= 0.15 * np.abs(r).max() + 1e-7, (i, lay, size)
                 off += size
         cos = float(got[i] @ g / (np.linalg.norm(got[i]) * np.linalg.norm(g)))
         assert cos > 0.995, cos
         assert abs(float(loss[i]) - le) <= 1e-4 * max(abs(le), 1.0)
         assert abs(float(loss[i]) - l) <= 2e-2 * max(abs(l), 1.0)
-    print("bf16 gradient vs bf16-point reference: worst block-relative error %.2e" % worst)
+    print("bf16 gradient vs bf16-point reference: worst block 2-norm error %.2e" % worst)
     assert np.count_nonzero(G.cpu().numpy()) <= m.d * n     # padding untouched
     h.close()
 
@@ -510,7 +516,8 @@ def test_mix_with_a_mask_that_disagrees_with_b(rule):
 
 
 @pytest.mark.parametrize("kernel,graph,panel", [("mix_panel_kernel", "reg4_32", 0), ("mix_staged_kernel", "reg32_256", 1),
-                                                ("mix_direct_kernel", "reg4_32", -1), ("mix_tc_kernel", "reg32_256", 2)])
+                                                ("mix_direct_kernel", "reg4_32", -1), ("mix_tc_kernel", "reg32_256", 2),
+                                                ("mix_sp_kernel", "reg32_256", 3)])
 @pytest.mark.parametrize("order", ["local_then_mix", "mix_then_correct"])
 def test_consensus_only_mix_reads_no_gradient(kernel, graph, panel, order):
     """G == NULL (Section 3.2.1's truncated model: gradients zero after K) gives the bits of a mix with an
