@@ -217,6 +217,19 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
               float* loss, void* stream);
 
 /*
+ * Single-launch round (Algorithm 1, one iteration, as ONE cooperative kernel launch).  For networks whose
+ * round is bound by launch latency (an fp32 model and at most 64 workers) dbw_round with batch_idx runs
+ * gather, forward, loss, backward, selection, weights, times and the mix inside one persistent kernel with
+ * grid-wide barriers between dependent steps.  The results are bit-identical to the multi-launch path (the
+ * same device functions in the same order per output element).  On by default where it applies;
+ * dbw_set_fused_round(h, 0) returns to one launch per step.  dbw_round_is_fused() tells which path
+ * dbw_round would take (1 = single launch).  With stage timing on, the whole launch is reported under
+ * stage 0.
+ */
+int dbw_set_fused_round(dbw_handle* h, int enable);
+int dbw_round_is_fused(const dbw_handle* h);
+
+/*
  * Parameter tracking for chained rounds (tensor-core path; a no-op otherwise).  Each round the
  * BF16 GEMMs need a bf16 copy of the weights.  With tracking on, dbw_mix / dbw_round write that copy
  * next to X' (same values as a later cast, so results do not change), and the next dbw_grad /

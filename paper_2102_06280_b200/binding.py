@@ -56,6 +56,8 @@ _SIGNATURES = {
     "dbw_set_mix_panel": (C.c_int, [_P, C.c_int32]),
     "dbw_mix_kernel": (C.c_int, [_P]),
     "dbw_set_param_tracking": (C.c_int, [_P, C.c_int]),
+    "dbw_set_fused_round": (C.c_int, [_P, C.c_int]),
+    "dbw_round_is_fused": (C.c_int, [_P]),
     "dbw_round": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_round_host": (C.c_int, [_P, _P, _P, _P, _P, _P, C.c_float, _P, _P, _P, _P, _P, _P, _P]),
     "dbw_update_backups": (C.c_int, [_P, _P, _P, _P, _P]),
@@ -213,6 +215,12 @@ class Dbw:
 
     def set_param_tracking(self, enable: bool):
         _check(lib().dbw_set_param_tracking(self._h, int(bool(enable))), "dbw_set_param_tracking")
+
+    def set_fused_round(self, enable: bool):
+        _check(lib().dbw_set_fused_round(self._h, int(bool(enable))), "dbw_set_fused_round")
+
+    def round_is_fused(self) -> bool:
+        return bool(_check(lib().dbw_round_is_fused(self._h), "dbw_round_is_fused"))
 
     def mix_kernel(self) -> str:
         return ("mix_direct_kernel", "mix_panel_kernel", "mix_staged_kernel", "mix_tc_kernel", "mix_sp_kernel")[_check(lib().dbw_mix_kernel(self._h), "dbw_mix_kernel")]

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdbw.so")
-SOURCES = ["api.cu", "select.cu", "mix.cu", "mix_staged.cu", "mix_tc.cu", "mix_sp.cu", "dtur.cu", "grad_fp32.cu", "grad_bf16.cu", "probe.cu"]
+SOURCES = ["api.cu", "select.cu", "mix.cu", "mix_staged.cu", "mix_tc.cu", "mix_sp.cu", "dtur.cu", "grad_fp32.cu", "grad_bf16.cu", "round_fused.cu", "probe.cu"]
 
 
 def _nvcc() -> str:

@@ -121,6 +121,7 @@ void free_all(dbw_handle* h) {
     grad_bf16_free(h);
     mix_tc_free(h);
     mix_sp_free(h);
+    round_fused_free(h);
     void* ptrs[] = {h->d_rowptr, h->d_col, h->d_links, h->d_covered, h->d_epoch, h->d_status, h->d_waited,
                     h->d_ticket, h->d_Tnbr_ws, h->plan.idx, h->plan.w, h->plan.w_self, h->plan.cnt, h->d_G,
                     h->s_t, h->s_b, h->s_bidx, h->s_kept, h->s_Tw, h->s_Tr, h->s_loss};
@@ -247,6 +248,7 @@ int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* 
         h->model = *model;
         rc = (flags & DBW_GEMM_BF16) ? grad_bf16_alloc(h) : grad_fp32_alloc(h);
         if (rc) return fail(rc);
+        round_fused_prepare(h);  // the single-launch round, for the networks it serves
     }
     *out = h;
     return DBW_OK;
@@ -321,6 +323,14 @@ int dbw_set_param_tracking(dbw_handle* h, int enable) {
     return DBW_OK;
 }
 
+int dbw_set_fused_round(dbw_handle* h, int enable) {
+    if (!h) return DBW_ERR_NULL;
+    h->fused_enabled = enable != 0;
+    return DBW_OK;
+}
+
+int dbw_round_is_fused(const dbw_handle* h) { return h ? (round_fused_usable(h) ? 1 : 0) : DBW_ERR_NULL; }
+
 int dbw_mix_in_place_ok(const dbw_handle* h) { return h && mix_panel_fits(h) ? 1 : 0; }
 
 int dbw_mix_kernel(const dbw_handle* h) { return h ? mix_kernel_kind(h) : DBW_ERR_NULL; }
@@ -354,6 +364,15 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
             h->prof_events.push_back(e);
         }
         ev = &h->prof_events[6 * h->prof_rounds++];
+    }
+    if (batch_idx && round_fused_usable(h)) {
+        // small fp32 network: the whole iteration in one cooperative launch (same bits as the launches below)
+        if (ev) DBW_CUDA(cudaEventRecord(ev[0], s));
+        rc = launch_round_fused(h, X, t, b, batch_idx, lr, lr_per_worker, X_out, kept, T_worker, T_nbr, T_round, loss, s);
+        if (ev)
+            for (int e = 1; e < 6; ++e) DBW_CUDA(cudaEventRecord(ev[e], s));  // the stages are not separable: all under "gradients"
+        h->shadow_valid = false;
+        return rc;
     }
     // first error of the calls below; later calls still run so that a forked side stream is always joined
     int first = DBW_OK;

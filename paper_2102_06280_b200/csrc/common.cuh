@@ -65,6 +65,7 @@ struct MixPlan {
 struct BF16State;  // tensor-core gradient path (grad_bf16.cu)
 struct TcMixState;  // tensor-core mix (mix_tc.cu)
 struct SpMixState;  // tensor-core mix with 2:4 structured sparsity (mix_sp.cu)
+struct FusedState;  // single-launch round for small networks (round_fused.cu)
 
 }  // namespace dbw
 
@@ -98,6 +99,9 @@ struct dbw_handle {
     int mix_panel_cols = 0;  // 0 = automatic
     dbw::TcMixState* mix_tc = nullptr;  // selection matrix and tensor map of the tensor-core mix (lazy)
     dbw::SpMixState* mix_sp = nullptr;  // 2:4 order, compressed selection matrix and tensor maps of the sparse tensor-core mix (dbw_init)
+
+    dbw::FusedState* fused = nullptr;   // single-launch round (dbw_init); used by dbw_round while fused_enabled
+    bool fused_enabled = true;
 
     // model / gradient path
     bool has_model = false;
@@ -178,6 +182,14 @@ void mix_sp_free(dbw_handle* h);
 int launch_mix_sp(dbw_handle* h, const float* X, const float* G, float lr, const float* lr_pw, float* X_out,
                   uint16_t* shadow, cudaStream_t s);
 int mix_sp_order_host(int N, const int32_t* rowptr, const int32_t* col, int32_t* order, int capacity);
+
+// round_fused.cu
+void round_fused_prepare(dbw_handle* h);
+bool round_fused_usable(const dbw_handle* h);
+void round_fused_free(dbw_handle* h);
+int launch_round_fused(dbw_handle* h, const float* X, const double* t, const int32_t* b, const int32_t* batch_idx, float lr,
+                       const float* lr_pw, float* X_out, uint8_t* kept, double* T_worker, double* T_nbr, double* T_round,
+                       float* loss, cudaStream_t s);
 
 // dtur.cu
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);

@@ -2,196 +2,39 @@
 // CUDA cores, for all workers at once: every kernel is batched over workers (blockIdx.z), whose
 // weights are slices of their rows of X.
 #include "common.cuh"
+#include "round_dev.cuh"
 
 namespace dbw {
 
 namespace {
 
-// ------------------------------------------------------------------ batch gather
-// A sample index outside [0, S) or a label outside [0, C) is clamped and reported in the status word.
+using namespace dev;
+
+// ------------------------------------------------------------------ kernels (bodies in round_dev.cuh)
 __global__ void gather_batch_kernel(int B, int S, int in_dim, int C, const float* __restrict__ feat,
                                     const int32_t* __restrict__ labels, const int32_t* __restrict__ batch_idx,
                                     float* __restrict__ A0, int32_t* __restrict__ ylab, uint32_t* status) {
-    const int s = blockIdx.x, i = blockIdx.y;
-    int src = batch_idx[(size_t)i * B + s];
-    if (src < 0 || src >= S) {
-        if (threadIdx.x == 0) atomicOr(status, DBW_STATUS_BAD_INDEX);
-        src = src < 0 ? 0 : S - 1;
-    }
-    const float* from = feat + ((size_t)i * S + src) * in_dim;
-    float* to = A0 + ((size_t)i * B + s) * in_dim;
-    if ((in_dim & 3) == 0) {
-        for (int k = threadIdx.x; k < in_dim / 4; k += blockDim.x)
-            reinterpret_cast<float4*>(to)[k] = __ldg(reinterpret_cast<const float4*>(from) + k);
-    } else {
-        for (int k = threadIdx.x; k < in_dim; k += blockDim.x) to[k] = from[k];
-    }
-    if (threadIdx.x == 0) {
-        int y = labels[(size_t)i * S + src];
-        if (y < 0 || y >= C) {
-            atomicOr(status, DBW_STATUS_BAD_INDEX);
-            y = y < 0 ? 0 : C - 1;
-        }
-        ylab[(size_t)i * B + s] = y;
-    }
+    gather_row(blockIdx.x, blockIdx.y, B, S, in_dim, C, feat, labels, batch_idx, A0, ylab, status);
 }
 
-// ------------------------------------------------------------------ batched strided GEMM
-// C[z][m][n] = epilogue( sum_k A[z](m,k) * B[z](k,n) ), operands addressed through strides so
-// that the same kernel serves Z = A W^T, dW = dZ^T A and dA = dZ W.
-struct GemmArgs {
-    const float* A;
-    long long sAz, sAm, sAk;
-    const float* B;
-    long long sBz, sBn, sBk;
-    float* C;
-    long long sCz, sCm;
-    const float* bias;  // indexed by n, nullable
-    long long sBiasz;
-    const float* mask;  // same shape as C, nullable: C *= (mask > 0)
-    long long sMz, sMm;
-    int M, N, K;
-    int relu;
-};
-
-
-// 256 threads, each an R x R micro-tile: tiles of 64 x 64 (R = 4) for large outputs, 32 x 32 (R = 2)
-// when the larger tile would leave most SMs idle.  TK = depth of one k-step: 16, or 64 for the few-CTA
-// case with a long reduction, where a step costs one global-memory round trip whatever its depth
-// (the order of the additions is the same).
 template <int R, int TK>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
-    constexpr int T = 16 * R;        // tile edge
-    constexpr int PER = T * TK / 256;  // elements of each operand tile a thread stages
+    constexpr int T = 16 * R;
     __shared__ __align__(16) float As[TK][T + 4];
     __shared__ __align__(16) float Bs[TK][T + 4];
-    const int z = blockIdx.z;
-    const int m0 = blockIdx.y * T, n0 = blockIdx.x * T;
-    const float* A = g.A + (size_t)z * g.sAz;
-    const float* B = g.B + (size_t)z * g.sBz;
-    const int tid = threadIdx.x;
-    const int tx = tid & 15, ty = tid >> 4;
-    const bool a_k_fast = g.sAk == 1;
-    const bool b_k_fast = g.sBk == 1;
-    float acc[R][R] = {};
-    float pa[PER], pb[PER];  // next k-step's operand elements, in flight while this one is multiplied
-    auto fetch = [&](int k0) {
-#pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const int e = tid + r * 256;
-            const int ka = a_k_fast ? (e % TK) : (e / T);
-            const int ma = a_k_fast ? (e / TK) : (e % T);
-            pa[r] = (m0 + ma < g.M && k0 + ka < g.K) ? __ldg(A + (size_t)(m0 + ma) * g.sAm + (size_t)(k0 + ka) * g.sAk) : 0.f;
-            const int kb = b_k_fast ? (e % TK) : (e / T);
-            const int nb = b_k_fast ? (e / TK) : (e % T);
-            pb[r] = (n0 + nb < g.N && k0 + kb < g.K) ? __ldg(B + (size_t)(n0 + nb) * g.sBn + (size_t)(k0 + kb) * g.sBk) : 0.f;
-        }
-    };
-    fetch(0);
-    for (int k0 = 0; k0 < g.K; k0 += TK) {
-#pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const int e = tid + r * 256;
-            As[a_k_fast ? (e % TK) : (e / T)][a_k_fast ? (e / TK) : (e % T)] = pa[r];
-            Bs[b_k_fast ? (e % TK) : (e / T)][b_k_fast ? (e / TK) : (e % T)] = pb[r];
-        }
-        __syncthreads();
-        fetch(k0 + TK);  // all zero past the end
-#pragma unroll
-        for (int kk = 0; kk < TK; ++kk) {
-            float av[R], bv[R];
-            if constexpr (R == 4) {  // one 128-bit shared load per operand (rows are 16-byte aligned: T + 4 = 68 floats)
-                const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-                const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-                av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
-                bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
-            } else {
-                const float2 a2 = *reinterpret_cast<const float2*>(&As[kk][ty * 2]);
-                const float2 b2 = *reinterpret_cast<const float2*>(&Bs[kk][tx * 2]);
-                av[0] = a2.x; av[1] = a2.y;
-                bv[0] = b2.x; bv[1] = b2.y;
-            }
-#pragma unroll
-            for (int i = 0; i < R; ++i)
-#pragma unroll
-                for (int j = 0; j < R; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-    float* C = g.C + (size_t)z * g.sCz;
-    const float* bias = g.bias ? g.bias + (size_t)z * g.sBiasz : nullptr;
-    const float* mask = g.mask ? g.mask + (size_t)z * g.sMz : nullptr;
-#pragma unroll
-    for (int i = 0; i < R; ++i) {
-        const int m = m0 + ty * R + i;
-        if (m >= g.M) continue;
-#pragma unroll
-        for (int j = 0; j < R; ++j) {
-            const int n = n0 + tx * R + j;
-            if (n >= g.N) continue;
-            float v = acc[i][j];
-            if (bias) v += bias[n];
-            if (g.relu) v = fmaxf(v, 0.f);
-            if (mask && !(mask[(size_t)m * g.sMm + n] > 0.f)) v = 0.f;
-            C[(size_t)m * g.sCm + n] = v;
-        }
-    }
+    gemm_tile<R, TK>(g, blockIdx.z, blockIdx.y * T, blockIdx.x * T, As, Bs);
 }
 
-// ------------------------------------------------------------------ softmax cross-entropy
-// One CTA per worker, one warp per sample at a time.  dZ = (softmax(z) - onehot(y)) / B;
-// loss = mean over the batch of (logsumexp(z) - z_y), summed in a fixed order.  The CTA then also sums
-// its worker's dZ over the batch: the bias gradient of the last layer (one launch less per round).
 __global__ void __launch_bounds__(256)
 softmax_ce_kernel(int B, int C, const float* __restrict__ logits, const int32_t* __restrict__ ylab,
                   float* dz, float* __restrict__ loss, float* __restrict__ G, long long ld, long long b_off) {
-    const int i = blockIdx.x;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float invB = 1.0f / (float)B;
-    float wloss = 0.f;
-    for (int s = warp; s < B; s += 8) {
-        const float* z = logits + ((size_t)i * B + s) * C;
-        float* o = dz + ((size_t)i * B + s) * C;
-        const int y = ylab[(size_t)i * B + s];
-        float mx = -INFINITY;
-        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
-#pragma unroll
-        for (int k = 16; k > 0; k >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, k));
-        float sum = 0.f;
-        for (int c = lane; c < C; c += 32) sum += expf(z[c] - mx);
-#pragma unroll
-        for (int k = 16; k > 0; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
-        const float inv = 1.0f / sum;
-        for (int c = lane; c < C; c += 32) o[c] = (expf(z[c] - mx) * inv - (c == y ? 1.f : 0.f)) * invB;
-        wloss += (mx + logf(sum)) - z[y];
-    }
     __shared__ float sl[8];
-    if (lane == 0) sl[warp] = wloss;
-    __syncthreads();
-    if (threadIdx.x == 0 && loss) {
-        float t = 0.f;
-        for (int w = 0; w < 8; ++w) t += sl[w];
-        loss[i] = t * invB;
-    }
-    // db[c] = sum over the samples of dZ[s][c], in sample order (the barrier above ordered the dZ stores)
-    for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        const float* p = dz + (size_t)i * B * C + c;
-        float t = 0.f;
-        for (int s = 0; s < B; ++s) t += p[(size_t)s * C];
-        G[(size_t)i * ld + b_off + c] = t;
-    }
+    softmax_ce_worker(blockIdx.x, B, C, logits, ylab, dz, loss, G, ld, b_off, sl);
 }
 
-// db[z][o] = sum_m dZ[z][m][o]
 __global__ void bias_grad_kernel(int B, int out_dim, const float* __restrict__ dz, float* __restrict__ G,
                                  long long ld, long long b_off) {
-    const int i = blockIdx.y;
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= out_dim) return;
-    const float* p = dz + (size_t)i * B * out_dim + o;
-    float s = 0.f;
-    for (int m = 0; m < B; ++m) s += p[(size_t)m * out_dim];
-    G[(size_t)i * ld + b_off + o] = s;
+    bias_grad_col(blockIdx.y, blockIdx.x * blockDim.x + threadIdx.x, B, out_dim, dz, G, ld, b_off);
 }
 
 int run_gemm(const GemmArgs& g, int batch, int sm_count, cudaStream_t s) {

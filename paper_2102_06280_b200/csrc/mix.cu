@@ -9,6 +9,7 @@
 // G == nullptr in any of the kernels means G = 0 (a consensus-only round): nothing of G is read, 8 bytes
 // per element.
 #include "common.cuh"
+#include "round_dev.cuh"
 
 namespace dbw {
 
@@ -16,15 +17,7 @@ namespace {
 
 constexpr int kMixThreads = 512;
 
-__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
-
-__device__ __forceinline__ float4 fma4(float w, float4 v, float4 a) {
-    a.x = fmaf(w, v.x, a.x);
-    a.y = fmaf(w, v.y, a.y);
-    a.z = fmaf(w, v.z, a.z);
-    a.w = fmaf(w, v.w, a.w);
-    return a;
-}
+using namespace dev;
 
 template <int GS>
 __global__ void __launch_bounds__(kMixThreads, 3)
@@ -32,57 +25,8 @@ mix_panel_kernel(int N, long long ld, const float* X, const float* __restrict__ 
                  const float* __restrict__ lr_pw, float* Xout, uint16_t* __restrict__ shadow, MixPlan plan,
                  int mix_then_correct, int n_panels) {
     extern __shared__ float4 sm[];  // [N][GS]
-    const int tid = threadIdx.x;
-    const int q = tid % GS;
-    const int gid = tid / GS;
-    constexpr int kGroups = kMixThreads / GS;
-    const int total = N * GS;
-
     for (int panel = blockIdx.x; panel < n_panels; panel += gridDim.x) {
-        const long long col0 = (long long)panel * (4 * GS);
-        // ---- stage the panel: x (Eq. 3 order) or x - lr*g (Eq. 4) ----
-#pragma unroll 4
-        for (int idx = tid; idx < total; idx += kMixThreads) {
-            const int r = idx / GS;
-            const long long c = col0 + 4 * (idx % GS);
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c < ld) {
-                v = ldg4(X + (size_t)r * ld + c);
-                if (G && !mix_then_correct) {
-                    const float4 g = ldg4(G + (size_t)r * ld + c);
-                    const float nlr = -(lr_pw ? lr_pw[r] : lr);
-                    v = fma4(nlr, g, v);
-                }
-            }
-            sm[idx] = v;
-        }
-        __syncthreads();
-        // ---- every output row of the panel ----
-        const long long c = col0 + 4 * q;
-        for (int i = gid; i < N; i += kGroups) {
-            const float ws = plan.w_self[i];
-            const float4 self = sm[i * GS + q];
-            float4 acc = make_float4(ws * self.x, ws * self.y, ws * self.z, ws * self.w);
-            const int cnt = plan.cnt[i];
-            const int4* pi = reinterpret_cast<const int4*>(plan.idx + (size_t)i * plan.stride);
-            const float4* pw = reinterpret_cast<const float4*>(plan.w + (size_t)i * plan.stride);
-            for (int k = 0; k < cnt; k += 4) {
-                const int4 j = __ldg(pi + (k >> 2));
-                const float4 w = __ldg(pw + (k >> 2));
-                acc = fma4(w.x, sm[j.x * GS + q], acc);
-                acc = fma4(w.y, sm[j.y * GS + q], acc);
-                acc = fma4(w.z, sm[j.z * GS + q], acc);
-                acc = fma4(w.w, sm[j.w * GS + q], acc);
-            }
-            if (c < ld) {
-                if (G && mix_then_correct) {
-                    const float4 g = ldg4(G + (size_t)i * ld + c);
-                    acc = fma4(-(lr_pw ? lr_pw[i] : lr), g, acc);
-                }
-                *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
-                if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);
-            }
-        }
+        mix_panel_body<GS, kMixThreads>(panel, sm, N, ld, X, G, lr, lr_pw, Xout, shadow, plan, mix_then_correct);
         __syncthreads();
     }
 }

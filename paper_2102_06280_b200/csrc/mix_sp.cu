@@ -21,7 +21,7 @@
 // of two row tiles (2 x 224 columns; CTA r of the pair holds rows 256 t + 128 r .. + 127 of tile t) and,
 // in its last 64 columns, the sparsity metadata of its 256 rows for all inputs (written once per launch).
 //   warp 0      TMA: compressed S tiles (128 rows x 128 inputs = 64 values, K-major, 128-byte swizzle) out
-//               of L2, 2-stage ring; L2 prefetch of the X and G row segments a few steps ahead
+//               of L2, 2-stage ring
 //   warp 1      MMA issue (leader CTA) + tensor-memory allocation (both CTAs)
 //   warps 2-5   metadata into tensor memory (once), then the epilogue: tcgen05.ld, row scale,
 //               128-byte-swizzled 32 x 32 blocks in shared memory, TMA stores
@@ -62,7 +62,6 @@ constexpr int kMetaCol = kTiles * kPanel;                    // first metadata c
 constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kAStages * kAStageBytes + (size_t)kBStages * kBStageBytes +
                               (size_t)kStagingBytes + 256 /*barriers*/;
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr int kPrefetchAhead = 6;  // piece stages of X and G rows requested into L2 ahead of the producers
 // kind::f16, sparse: D = f32, A = B = bf16, A K-major (compressed), B MN-major, N = 224, M = 256 (two CTAs)
 constexpr uint32_t kIdesc = (1u << 2) | (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kPanel >> 3) << 17) |
                             ((uint32_t)(256 >> 4) << 24);
@@ -115,10 +114,6 @@ __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* m
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
         : "memory");
-}
-// asks for `bytes` (a multiple of 16, from a 16-byte aligned address) to be brought into L2
-__device__ __forceinline__ void l2_prefetch(const void* p, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 // Arrives on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far are complete
 // (a barrier arrive sent to the two CTAs of the pair; no data moves).
@@ -264,26 +259,11 @@ mix_sp_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
     }
 
     if (warp == 0) {
-        // ---------------- compressed S tiles by TMA; X and G row segments prefetched into L2 ----------------
-        const int total_kb = my_items * n_kb;
-        auto prefetch = [&](int kb_global) {  // this CTA's 112 columns of the 32 rows of piece stage kb_global: one row per lane
-            if (kb_global >= total_kb) return;
-            const int w = kb_global / n_kb, kb = kb_global % n_kb;
-            const long long col = (long long)(group + w * groups) * kPanel + (long long)rank * kHalf;
-            if (col >= a.ld) return;
-            const int row = a.order[kb * kKB + lane];
-            if (row < 0) return;
-            const long long rem = a.ld - col;
-            const uint32_t bytes = (uint32_t)(rem < kHalf ? rem : kHalf) * 4u;
-            l2_prefetch(a.X + (size_t)row * a.ld + col, bytes);
-            if (a.G && !a.mix_then_correct) l2_prefetch(a.G + (size_t)row * a.ld + col, bytes);
-        };
-        for (int kb = 0; kb < kPrefetchAhead; ++kb) prefetch(kb);
+        // ---------------- compressed S tiles by TMA ----------------
         int it = 0;
         bool live = true;
         for (int w = 0; w < my_items && live; ++w)
             for (int ka = 0; ka < a.n_ka; ++ka, ++it) {
-                for (int sub = 0; sub < kKA / kKB; ++sub) prefetch(it * (kKA / kKB) + sub + kPrefetchAhead);
                 const int s = it % kAStages;
                 bool ok = true;
                 if (lane == 0 && it >= kAStages) ok = mbar_wait_paused(&bars->a_empty[s], ((it / kAStages) - 1) & 1, wc, 64);

@@ -1,6 +1,7 @@
 // Fastest-neighbour selection (Section 2.2), iteration times (Section 3.2.2) and the per-round
 // mixing plan with the weights of Assumption 1.  One warp per worker.
 #include "common.cuh"
+#include "round_dev.cuh"
 
 namespace dbw {
 
@@ -8,69 +9,10 @@ namespace {
 
 constexpr int kWarpsPerBlock = 4;
 
-// Arrival time used for ordering: NaN sorts last (as +inf) and is reported in the status word.
-__device__ __forceinline__ double order_time(double t, uint32_t* status) {
-    if (t != t) {
-        atomicOr(status, DBW_STATUS_NAN_TIME);
-        return __longlong_as_double(0x7ff0000000000000LL);
-    }
-    return t;
-}
+using namespace dev;
 
-__device__ __forceinline__ int clamped_b(const int32_t* b, int i, int deg, uint32_t* status) {
-    int bi = b[i];
-    if (bi < 0 || bi > deg) {
-        atomicOr(status, DBW_STATUS_BAD_B);
-        bi = bi < 0 ? 0 : deg;
-    }
-    return bi;
-}
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-__device__ __forceinline__ double warp_max(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-
-// Writes the compacted kept list of worker i (and its weights) given the per-lane keep decision
-// of one 32-neighbour chunk.  `running` is the number of entries already written.
-__device__ __forceinline__ void plan_append(const MixPlan& plan, int i, int lane, bool keep, int j, float w,
-                                            int& running) {
-    unsigned m = __ballot_sync(0xffffffffu, keep);
-    if (keep) {
-        int pos = running + __popc(m & ((1u << lane) - 1u));
-        plan.idx[(size_t)i * plan.stride + pos] = j;
-        plan.w[(size_t)i * plan.stride + pos] = w;
-    }
-    running += __popc(m);
-}
-
-__device__ __forceinline__ void plan_finish(const MixPlan& plan, int i, int lane, int cnt, float w_self) {
-    for (int k = cnt + lane; k < plan.stride; k += 32) {
-        plan.idx[(size_t)i * plan.stride + k] = i;
-        plan.w[(size_t)i * plan.stride + k] = 0.f;
-    }
-    if (lane == 0) {
-        plan.cnt[i] = cnt;
-        plan.w_self[i] = w_self;
-    }
-}
-
-__device__ __forceinline__ float edge_weight(bool uniform, int p_i, int p_j) {
-    int m = uniform ? p_i : (p_i > p_j ? p_i : p_j);
-    return 1.0f / (1.0f + (float)m);
-}
-
-// Selection: lane l of the warp owns neighbour (base + l) of worker i; its rank is the number of
-// neighbours whose (time, index) key is smaller, counted by shuffling every key past every lane.
-// A neighbour is kept when its rank is below p_i.  The last block to finish computes the
-// per-worker and per-round times, which need to know who is waited for by whom.
+// Selection: one warp per worker (dev::select_worker); the last block to finish computes the per-worker and
+// per-round times, which need to know who is waited for by whom.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
               const double* __restrict__ t, const double* __restrict__ t_edge, const int32_t* __restrict__ b,
@@ -80,53 +22,7 @@ select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restri
               int uniform) {
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    if (i < N) {
-        const int lo = rowptr[i], hi = rowptr[i + 1], deg = hi - lo;
-        const int p = deg - clamped_b(b, i, deg, status);
-        double tn = 0.0;
-        float wsum = 0.f;
-        int running = 0;
-        for (int base = 0; base < deg; base += 32) {
-            const int e = lo + base + lane;
-            const bool valid = e < hi;
-            const int j = valid ? col[e] : 0x7fffffff;
-            // arrival of col[e]'s update at worker i: the sender's time, or the link's own time
-            const double tj = valid ? order_time(t_edge ? t_edge[e] : t[j], status) : 0.0;
-            int rank = 0;
-            for (int base2 = 0; base2 < deg; base2 += 32) {
-                const int e2 = lo + base2 + lane;
-                const int j2 = e2 < hi ? col[e2] : 0x7fffffff;
-                const double t2 = e2 < hi ? order_time(t_edge ? t_edge[e2] : t[j2], status) : 0.0;
-                const int n2 = min(32, deg - base2);
-                for (int s = 0; s < n2; ++s) {
-                    const double ts = __shfl_sync(0xffffffffu, t2, s);
-                    const int js = __shfl_sync(0xffffffffu, j2, s);
-                    rank += (ts < tj) || (ts == tj && js < j);
-                }
-            }
-            const bool keep = valid && rank < p;
-            if (valid) kept[e] = keep ? 1 : 0;
-            if (keep) {
-                waited[j] = 1u;
-                tn = fmax(tn, tj);
-            }
-            if (build_plan) {
-                float w = 0.f;
-                if (keep) {
-                    const int dj = rowptr[j + 1] - rowptr[j];
-                    w = edge_weight(uniform, p, dj - clamped_b(b, j, dj, status));
-                    wsum += w;
-                }
-                plan_append(plan, i, lane, keep, j, w, running);
-            }
-        }
-        tn = warp_max(tn);
-        if (lane == 0) T_nbr_ws[i] = tn;
-        if (build_plan) {
-            wsum = warp_sum(wsum);
-            plan_finish(plan, i, lane, running, uniform ? 1.0f / (1.0f + (float)p) : 1.0f - wsum);
-        }
-    }
+    if (i < N) select_worker(i, lane, rowptr, col, t, t_edge, b, kept, T_nbr_ws, waited, status, plan, build_plan, uniform);
 
     // ---- last block: T_worker, T_round ----
     __shared__ bool is_last;
@@ -137,21 +33,7 @@ select_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restri
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    double tr = 0.0;
-    for (int w = threadIdx.x; w < N; w += blockDim.x) {
-        const int deg = rowptr[w + 1] - rowptr[w];
-        int bw = b[w];
-        bw = bw < 0 ? 0 : (bw > deg ? deg : bw);
-        const int p = deg - bw;
-        const bool part = p >= 1 || __ldcg(&waited[w]) != 0u;
-        const double tw = order_time(t[w], status);
-        const double tn = __ldcg(&T_nbr_ws[w]);
-        if (T_nbr_out) T_nbr_out[w] = tn;
-        const double twk = p >= 1 ? fmax(tw, tn) : (part ? tw : 0.0);
-        if (T_worker) T_worker[w] = twk;
-        if (part) tr = fmax(tr, twk);  // T(k) = max of T_j over the participating workers
-        waited[w] = 0u;
-    }
+    double tr = round_times_part(N, rowptr, t, b, T_nbr_ws, T_nbr_out, T_worker, waited, status);
     tr = warp_max(tr);
     if (lane == 0) red[threadIdx.x >> 5] = tr;
     __syncthreads();

@@ -375,6 +375,48 @@ def test_round_replays_from_a_cuda_graph(cfg, flag):
     sim.h.close()
 
 
+@pytest.mark.parametrize("cfg", [0, 1])
+@pytest.mark.parametrize("order", ["local_then_mix", "mix_then_correct"])
+def test_single_launch_round_is_bit_identical_to_the_multi_launch_round(cfg, order):
+    """Small fp32 networks run the whole iteration of Algorithm 1 as one cooperative kernel launch.  It calls the
+    same device functions as the kernels of the multi-launch path, so parameters, losses, masks and times must be
+    the same bits; and it really is one launch per round."""
+    import paper_2102_06280_b200 as p
+    from paper_2102_06280_b200 import binding
+    w = wl.make_workload(cfg) if cfg == 0 else wl.make_workload(cfg, samples=400)
+    times = wl.arrival_times(w, 4)
+    lrw = dev((0.02 + 0.05 * np.random.default_rng(5).random(w.N)).astype(np.float32))
+    results = []
+    for fused in (True, False):
+        sim = Sim(w)
+        if order == "mix_then_correct":           # a handle with the other update order
+            sim.h.close()
+            sim.h = p.Dbw(w.rowptr, w.col, d=sim.m.d, model=sim.m, flags=p.ORDER_MIX_THEN_CORRECT)
+            sim.h.set_dataset(dev(sim.feat), dev(sim.labels), w.samples)
+        sim.h.set_fused_round(fused)
+        assert sim.h.round_is_fused() == fused
+        X = dev(sim.m.pack(sim.X0))
+        out = torch.empty_like(X)
+        per_round = []
+        for k in range(4):
+            sim.backups(k, times[k])
+            before = binding.launch_count()
+            if k == 3:                            # per-worker learning rates, out of place
+                sim.h.round(X, dev(times[k]), sim.b_d, 0.0, out, sim.kept, batch_idx=dev(wl.batch_indices(w, k)),
+                            lr_per_worker=lrw, T_worker=sim.Tw, T_nbr=sim.Tn, T_round=sim.Tr, loss=sim.loss)
+                torch.cuda.synchronize()
+                X = out
+            else:
+                sim.gpu_round(X, times[k], wl.batch_indices(w, k), X)
+            per_round.append(binding.launch_count() - before)
+        assert all(n == 1 for n in per_round) if fused else all(n > 1 for n in per_round)
+        results.append((X.clone(), sim.loss.clone(), sim.kept.clone(), sim.Tw.clone(), sim.Tn.clone(), sim.Tr.clone()))
+        assert sim.h.status() == 0
+        sim.h.close()
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
+
+
 @pytest.mark.parametrize("cfg,flag", [(1, 0), (2, 4)])
 def test_rounds_are_reproducible_bit_for_bit(cfg, flag):
     """No atomics on floating-point data and fixed summation orders: the same round run twice (fresh
