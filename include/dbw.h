@@ -221,10 +221,11 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b,
  * round is bound by launch latency (an fp32 model and at most 64 workers) dbw_round with batch_idx runs
  * gather, forward, loss, backward, selection, weights, times and the mix inside one persistent kernel with
  * grid-wide barriers between dependent steps.  The results are bit-identical to the multi-launch path (the
- * same device functions in the same order per output element).  On by default where it applies;
- * dbw_set_fused_round(h, 0) returns to one launch per step.  dbw_round_is_fused() tells which path
- * dbw_round would take (1 = single launch).  With stage timing on, the whole launch is reported under
- * stage 0.
+ * same device functions in the same order per output element).  enable = -1 (the default) uses it where it
+ * is the faster path (networks of up to about 6e7 multiply-adds per forward pass: above that the per-step
+ * kernels, which put more blocks on an SM than a cooperative grid can, win), 1 wherever it applies, 0 never.
+ * dbw_round_is_fused() tells which path dbw_round would take (1 = single launch).  With stage timing on, the
+ * whole launch is reported under stage 0.
  */
 int dbw_set_fused_round(dbw_handle* h, int enable);
 int dbw_round_is_fused(const dbw_handle* h);

@@ -216,8 +216,9 @@ class Dbw:
     def set_param_tracking(self, enable: bool):
         _check(lib().dbw_set_param_tracking(self._h, int(bool(enable))), "dbw_set_param_tracking")
 
-    def set_fused_round(self, enable: bool):
-        _check(lib().dbw_set_fused_round(self._h, int(bool(enable))), "dbw_set_fused_round")
+    def set_fused_round(self, enable):
+        """True / False, or None for the library's own choice."""
+        _check(lib().dbw_set_fused_round(self._h, -1 if enable is None else int(bool(enable))), "dbw_set_fused_round")
 
     def round_is_fused(self) -> bool:
         return bool(_check(lib().dbw_round_is_fused(self._h), "dbw_round_is_fused"))

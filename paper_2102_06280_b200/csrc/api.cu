@@ -325,7 +325,7 @@ int dbw_set_param_tracking(dbw_handle* h, int enable) {
 
 int dbw_set_fused_round(dbw_handle* h, int enable) {
     if (!h) return DBW_ERR_NULL;
-    h->fused_enabled = enable != 0;
+    h->fused_mode = enable < 0 ? -1 : (enable ? 1 : 0);
     return DBW_OK;
 }
 
@@ -364,13 +364,17 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
             h->prof_events.push_back(e);
         }
         ev = &h->prof_events[6 * h->prof_rounds++];
+        if ((int)h->prof_single.size() < h->prof_rounds) h->prof_single.resize(h->prof_rounds);
+        h->prof_single[h->prof_rounds - 1] = 0;
     }
     if (batch_idx && round_fused_usable(h)) {
         // small fp32 network: the whole iteration in one cooperative launch (same bits as the launches below)
         if (ev) DBW_CUDA(cudaEventRecord(ev[0], s));
         rc = launch_round_fused(h, X, t, b, batch_idx, lr, lr_per_worker, X_out, kept, T_worker, T_nbr, T_round, loss, s);
-        if (ev)
-            for (int e = 1; e < 6; ++e) DBW_CUDA(cudaEventRecord(ev[e], s));  // the stages are not separable: all under "gradients"
+        if (ev) {  // the stages are not separable: one pair of events, reported under "gradients"
+            DBW_CUDA(cudaEventRecord(ev[1], s));
+            h->prof_single[h->prof_rounds - 1] = 1;
+        }
         h->shadow_valid = false;
         return rc;
     }
@@ -421,6 +425,13 @@ int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds) {
     DeviceGuard guard(h->device);
     for (int r = 0; r < h->prof_rounds; ++r) {
         cudaEvent_t* ev = &h->prof_events[6 * r];
+        if (h->prof_single[r]) {  // a single-launch round: one pair of events
+            float v = 0.f;
+            DBW_CUDA(cudaEventSynchronize(ev[1]));
+            DBW_CUDA(cudaEventElapsedTime(&v, ev[0], ev[1]));
+            ms[0] += v;
+            continue;
+        }
         DBW_CUDA(cudaEventSynchronize(ev[5]));
         for (int st = 0; st < 3; ++st) {  // gradients, selection (beside the gradients when there are any), mix
             float v = 0.f;

@@ -100,8 +100,8 @@ struct dbw_handle {
     dbw::TcMixState* mix_tc = nullptr;  // selection matrix and tensor map of the tensor-core mix (lazy)
     dbw::SpMixState* mix_sp = nullptr;  // 2:4 order, compressed selection matrix and tensor maps of the sparse tensor-core mix (dbw_init)
 
-    dbw::FusedState* fused = nullptr;   // single-launch round (dbw_init); used by dbw_round while fused_enabled
-    bool fused_enabled = true;
+    dbw::FusedState* fused = nullptr;   // single-launch round (dbw_init)
+    int fused_mode = -1;                // -1 = where it is the faster path, 0 = never, 1 = wherever it applies
 
     // model / gradient path
     bool has_model = false;
@@ -130,6 +130,7 @@ struct dbw_handle {
     // stage timing (dbw_profile): events[round][0..5] = start / end of the gradient, selection and mix stages
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;
+    std::vector<char> prof_single;  // per recorded round: 1 = single-launch round (events 0 and 1 only)
     int prof_rounds = 0;
 
     // device staging of dbw_round_host

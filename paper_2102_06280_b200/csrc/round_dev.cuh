@@ -160,21 +160,51 @@ __device__ __forceinline__ void softmax_ce_worker(int i, int B, int C, const flo
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float invB = 1.0f / (float)B;
     float wloss = 0.f;
-    for (int s = warp; s < B; s += 8) {
-        const float* z = logits + ((size_t)i * B + s) * C;
-        float* o = dz + ((size_t)i * B + s) * C;
-        const int y = ylab[(size_t)i * B + s];
-        float mx = -INFINITY;
-        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+    if (C <= 32) {
+        // at most one class per lane: four samples of this warp per pass, their loads issued together (the
+        // arithmetic of each sample and the order in which the losses are added are those of the loop below)
+        for (int s0 = warp; s0 < B; s0 += 32) {
+            float zv[4];
+            int yv[4];
 #pragma unroll
-        for (int k = 16; k > 0; k >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, k));
-        float sum = 0.f;
-        for (int c = lane; c < C; c += 32) sum += expf(z[c] - mx);
+            for (int u = 0; u < 4; ++u) {
+                const int s = s0 + 8 * u;
+                zv[u] = (s < B && lane < C) ? logits[((size_t)i * B + s) * C + lane] : -INFINITY;
+                yv[u] = s < B ? ylab[(size_t)i * B + s] : 0;
+            }
 #pragma unroll
-        for (int k = 16; k > 0; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
-        const float inv = 1.0f / sum;
-        for (int c = lane; c < C; c += 32) o[c] = (expf(z[c] - mx) * inv - (c == y ? 1.f : 0.f)) * invB;
-        wloss += (mx + logf(sum)) - z[y];
+            for (int u = 0; u < 4; ++u) {
+                const int s = s0 + 8 * u;
+                if (s >= B) break;  // warp-uniform
+                float mx = zv[u];
+#pragma unroll
+                for (int k = 16; k > 0; k >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, k));
+                const float ez = lane < C ? expf(zv[u] - mx) : 0.f;
+                float sum = ez;
+#pragma unroll
+                for (int k = 16; k > 0; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+                const float inv = 1.0f / sum;
+                if (lane < C) dz[((size_t)i * B + s) * C + lane] = (ez * inv - (lane == yv[u] ? 1.f : 0.f)) * invB;
+                wloss += (mx + logf(sum)) - __shfl_sync(0xffffffffu, zv[u], yv[u] & 31);
+            }
+        }
+    } else {
+        for (int s = warp; s < B; s += 8) {
+            const float* z = logits + ((size_t)i * B + s) * C;
+            float* o = dz + ((size_t)i * B + s) * C;
+            const int y = ylab[(size_t)i * B + s];
+            float mx = -INFINITY;
+            for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+#pragma unroll
+            for (int k = 16; k > 0; k >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, k));
+            float sum = 0.f;
+            for (int c = lane; c < C; c += 32) sum += expf(z[c] - mx);
+#pragma unroll
+            for (int k = 16; k > 0; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+            const float inv = 1.0f / sum;
+            for (int c = lane; c < C; c += 32) o[c] = (expf(z[c] - mx) * inv - (c == y ? 1.f : 0.f)) * invB;
+            wloss += (mx + logf(sum)) - z[y];
+        }
     }
     if (lane == 0) sl[warp] = wloss;
     __syncthreads();
@@ -187,6 +217,7 @@ __device__ __forceinline__ void softmax_ce_worker(int i, int B, int C, const flo
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
         const float* p = dz + (size_t)i * B * C + c;
         float t = 0.f;
+#pragma unroll 8
         for (int s = 0; s < B; ++s) t += p[(size_t)s * C];
         G[(size_t)i * ld + b_off + c] = t;
     }
@@ -198,6 +229,7 @@ __device__ __forceinline__ void bias_grad_col(int i, int o, int B, int out_dim, 
     if (o >= out_dim) return;
     const float* p = dz + (size_t)i * B * out_dim + o;
     float s = 0.f;
+#pragma unroll 8
     for (int m = 0; m < B; ++m) s += p[(size_t)m * out_dim];
     G[(size_t)i * ld + b_off + o] = s;
 }

@@ -30,10 +30,12 @@ using namespace dev;
 constexpr int kThreads = 256;
 constexpr int kMixGS = 32;                       // 128-column panels
 constexpr int kMaxWorkers = 64;                  // N * kMixGS * 16 bytes of panel <= 32 KiB
-constexpr int kSmemBytes = 2 * 64 * 68 * 4;      // the largest GEMM staging (64 x 64 tiles, 64-deep steps): 34,816 bytes
+constexpr int kSmemBytes = 2 * 128 * 36 * 4;     // the largest GEMM staging (32 x 32 tiles, 128-deep steps): 36,864 bytes
+constexpr int kBlocksPerSM = 1;                  // registers are spent on deep k-steps (a step costs one memory round trip)
+constexpr long long kAutoMaxMacs = 64ll << 20;   // multiply-adds of the forward pass up to which the launch is used unasked
 
 // GEMM tile variants (R, TK) the kernel instantiates; which one a GEMM uses is chosen on the host.
-enum { V_2_16 = 0, V_2_64 = 1, V_4_16 = 2, V_4_64 = 3 };
+enum { V_2_16 = 0, V_2_64 = 1, V_4_16 = 2, V_4_64 = 3, V_2_128 = 4, kVariants = 5 };
 
 struct FusedArgs {
     int N, B, S, L, C;
@@ -87,11 +89,12 @@ __device__ __forceinline__ void gemm_any(int variant, const GemmArgs& g, int wor
         case V_2_16: gemm_tiles<2, 16>(g, workers, smem); break;
         case V_2_64: gemm_tiles<2, 64>(g, workers, smem); break;
         case V_4_16: gemm_tiles<4, 16>(g, workers, smem); break;
-        default: gemm_tiles<4, 64>(g, workers, smem); break;
+        case V_4_64: gemm_tiles<4, 64>(g, workers, smem); break;
+        default: gemm_tiles<2, 128>(g, workers, smem); break;  // a handful of tiles with a long reduction
     }
 }
 
-__global__ void __launch_bounds__(kThreads) round_fused_kernel(FusedArgs a) {
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(FusedArgs a) {
     extern __shared__ __align__(16) float smem[];
     __shared__ float sl[8];
     __shared__ double red[kThreads / 32];
@@ -175,10 +178,10 @@ __global__ void __launch_bounds__(kThreads) round_fused_kernel(FusedArgs a) {
 // Which tile variant a GEMM of `workers` problems M x N x K should take on a grid of `grid` blocks: the
 // one with the fewest waves x k-steps, a k-step costing a global-memory round trip plus its multiply-adds.
 int pick_variant(int M, int Nn, int K, int workers, int grid) {
-    const int Rs[4] = {2, 2, 4, 4}, TKs[4] = {16, 64, 16, 64};
+    const int Rs[kVariants] = {2, 2, 4, 4, 2}, TKs[kVariants] = {16, 64, 16, 64, 128};
     int best = 0;
     double best_cost = 1e300;
-    for (int v = 0; v < 4; ++v) {
+    for (int v = 0; v < kVariants; ++v) {
         const int T = 16 * Rs[v];
         const long long tiles = (long long)((M + T - 1) / T) * ((Nn + T - 1) / T) * workers;
         const long long waves = (tiles + grid - 1) / grid;
@@ -196,6 +199,7 @@ int pick_variant(int M, int Nn, int K, int workers, int grid) {
 
 struct FusedState {
     bool usable = false;
+    bool auto_on = false;
     int max_blocks = 0;
 };
 
@@ -214,11 +218,20 @@ void round_fused_prepare(dbw_handle* h) {
     int coop = 0, per_sm = 0;
     if (!cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device)) || !coop) return;
     if (!cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, round_fused_kernel, kThreads, kSmemBytes)) || per_sm < 1) return;
-    st->max_blocks = h->sm_count;  // one block per SM keeps the grid barrier cheap; the work is small
+    st->max_blocks = h->sm_count * std::min(per_sm, kBlocksPerSM);
+    long long macs = 0;
+    for (int l = 0; l < h->model.n_layers; ++l) macs += (long long)h->N * h->model.batch * h->model.dims[l] * h->model.dims[l + 1];
+    st->auto_on = macs <= kAutoMaxMacs;
     st->usable = true;
 }
 
-bool round_fused_usable(const dbw_handle* h) { return h->fused && h->fused->usable && h->fused_enabled && h->feat; }
+// Used when asked for, or, left to itself, for networks so small that launch latency is most of the round
+// (measured: above roughly 1e8 multiply-adds per round the per-step kernels, which fill the SMs with more
+// blocks than a cooperative grid can hold, are faster).
+bool round_fused_usable(const dbw_handle* h) {
+    if (!h->fused || !h->fused->usable || !h->feat || h->fused_mode == 0) return false;
+    return h->fused_mode > 0 || h->fused->auto_on;
+}
 
 int launch_round_fused(dbw_handle* h, const float* X, const double* t, const int32_t* b, const int32_t* batch_idx, float lr,
                        const float* lr_pw, float* X_out, uint8_t* kept, double* T_worker, double* T_nbr, double* T_round,
