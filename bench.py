@@ -55,7 +55,9 @@ def measured_peaks():
 class Job:
     """One workload resident on one GPU, stepped through the C ABI."""
 
-    def __init__(self, config: int, device: int = 0, rounds: int | None = None, **overrides):
+    def __init__(self, config: int, device: int = 0, rounds: int | None = None, col_range=None, **overrides):
+        """col_range = (c0, c1): this job owns only those columns of a mix-only workload's matrices (one column
+        shard of several; the update is independent per column, see paper_2102_06280_b200/sharding.py)."""
         import torch
         import paper_2102_06280_b200 as p
         self.torch, self.p = torch, p
@@ -85,16 +87,17 @@ class Job:
             self.ld = self.m.ld
         else:
             self.m = None
-            self.ld = w.d
-            self.h = p.Dbw(w.rowptr, w.col, d=w.d, ld=w.d, flags=flags, device=device)
-            self.X = torch.empty((w.N, w.d), dtype=torch.float32, device=self.dev)
-            self.G = torch.empty((w.N, w.d), dtype=torch.float32, device=self.dev)
+            c0, c1 = col_range if col_range is not None else (0, w.d)
+            self.ld = c1 - c0
+            self.h = p.Dbw(w.rowptr, w.col, d=self.ld, ld=self.ld, flags=flags, device=device)
+            self.X = torch.empty((w.N, self.ld), dtype=torch.float32, device=self.dev)
+            self.G = torch.empty((w.N, self.ld), dtype=torch.float32, device=self.dev)
             step = 64
             for r0 in range(0, w.N, step):
                 rows = range(r0, min(w.N, r0 + step))
-                self.X[r0:r0 + step].copy_(torch.from_numpy(wl.gaussian_rows(w.init_seed, rows, w.d)))
-                self.G[r0:r0 + step].copy_(torch.from_numpy(
-                    wl.gaussian_rows(wl.external_gradient_seed(w), rows, w.d, scale=0.01)))
+                self.X[r0:r0 + step].copy_(torch.from_numpy(np.ascontiguousarray(wl.gaussian_rows(w.init_seed, rows, w.d)[:, c0:c1])))
+                self.G[r0:r0 + step].copy_(torch.from_numpy(np.ascontiguousarray(
+                    wl.gaussian_rows(wl.external_gradient_seed(w), rows, w.d, scale=0.01)[:, c0:c1])))
             self.h_idx = self.d_idx = None
         self.h_t = torch.from_numpy(wl.arrival_times(w, self.n_rounds)).pin_memory()
         self.d_t = self.h_t.to(self.dev)
@@ -353,9 +356,10 @@ def max_over_ranks(ms, dist, device="cuda"):
     return float(tt.item())
 
 
-def aggregate_value(units_per_rank_step, steps, ms_max, world):
-    """Whole-job throughput of `world` replicas: all units processed / slowest rank's time."""
-    return world * units_per_rank_step * steps / (ms_max * 1e-3)
+def aggregate_value(units_per_rank_step, steps, ms_max, world, sharded=False):
+    """Whole-job throughput: `world` replicas (all units processed / slowest rank's time), or, column-sharded,
+    ONE simulation split over the ranks (its units / slowest rank's time)."""
+    return (1 if sharded else world) * units_per_rank_step * steps / (ms_max * 1e-3)
 
 
 def timed_loop(job, steps, fn, dist):
@@ -398,7 +402,14 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    res = measure(args.config, local, args, dist, overrides)
+    col_range = None
+    if args.shard == "columns":
+        from paper_2102_06280_b200.sharding import column_shards
+        full = wl.make_workload(args.config, **overrides)
+        if full.layers is not None:
+            raise SystemExit("--shard columns applies to the mix-only workloads (the gradients need whole rows)")
+        col_range = column_shards(full.d, world)[rank]
+    res = measure(args.config, local, args, dist, overrides, col_range)
     extra = {}
     # the whole hot path with a model (gradients on the tensor cores) next to the mix-only headline
     also = [c for c in (args.also or []) if c != args.config] if world == 1 and not overrides else []
@@ -411,7 +422,8 @@ def run_ours(args):
         return
     w = res["w"]
     line = {"metric": METRIC, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic"}
+            "higher_is_better": True, "scaling": "strong" if args.shard == "columns" else "weak", "vs_baseline": None,
+            "data": "synthetic"}
     line.update(summary(res, world, args))
     line["roofline"]["traffic"] = (MIX_TRAFFIC_BYTES.get(args.config)
                                    if not overrides and res["mix_kernel"] == "mix_staged_kernel" else None)
@@ -426,11 +438,11 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def measure(config, local, args, dist, overrides):
+def measure(config, local, args, dist, overrides, col_range=None):
     """Device-resident loop, stage times, launch count and the end-to-end loop of one workload."""
     import torch
     from paper_2102_06280_b200 import binding
-    job = Job(config, device=local, **overrides)
+    job = Job(config, device=local, col_range=col_range, **overrides)
     if args.mix_panel is not None:
         job.h.set_mix_panel(args.mix_panel)
     for _ in range(args.warmup):
@@ -478,16 +490,18 @@ def summary(res, world, args):
     mix_ms = res["stage_ms"]["mix"]
     achieved = res["mix_bytes"] / (mix_ms * 1e-3) / 1e9 if mix_ms > 0 else 0.0
     h2d, d2h = res["bytes"]
-    out = {"value": aggregate_value(w.N, args.steps, res["ms"], world), "ms_per_step": res["ms"] / args.steps,
+    sharded = getattr(args, "shard", "none") == "columns"
+    out = {"value": aggregate_value(w.N, args.steps, res["ms"], world, sharded), "ms_per_step": res["ms"] / args.steps,
            "dtype": "f32" if w.precision == "fp32" else "bf16",
            "config": {"workload": w.name, "N": w.N, "d": w.d, "ld": res["ld"], "nnz": int(len(w.col)),
                       "batch": w.batch, "layers": w.layers, "backups": w.backups, "weights": w.weight_rule,
                       "precision": "fp32" if w.precision == "fp32" else "bf16 operands, fp32 accumulate, fp32 master and mix",
                       "l2": "inputs larger than L2 (X and G each %.2f GB)" % (w.N * res["ld"] * 4 / 1e9)
                             if w.N * res["ld"] * 4 > 126e6 else "working set smaller than L2: cache-resident by design",
-                      "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+                      "multi_gpu": ("one simulation, X split by columns over %d ranks, no exchange (this rank: %d columns)" % (world, res["ld"])
+                                    if sharded else "replicas only" if world > 1 else "single GPU")},
            "stage_ms": res["stage_ms"],
-           "e2e": {"value": aggregate_value(w.N, args.steps, res["ms_e2e"], world), "unit": UNIT,
+           "e2e": {"value": aggregate_value(w.N, args.steps, res["ms_e2e"], world, sharded), "unit": UNIT,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": res["ms_e2e"] / args.steps},
            "gpu_launches": int(res["launches"]),
            "roofline": {"kernel": res["mix_kernel"], "bound": "hbm",
@@ -507,7 +521,7 @@ def summary(res, world, args):
         "peak_kind": "128 B/clk/SM x %d SMs x %.0f MHz (shared-memory data pipe, nominal)" % (res["sms"], peaks.get("sm_max_mhz", 1965.0))}
     if res.get("graph_ms"):
         out["cuda_graph"] = {"rounds_per_graph": args.graph, "ms_per_step": res["graph_ms"] / args.steps,
-                             "value": aggregate_value(w.N, args.steps, res["graph_ms"], world),
+                             "value": aggregate_value(w.N, args.steps, res["graph_ms"], world, sharded),
                              "note": "same rounds replayed from one CUDA graph per %d rounds" % args.graph}
     flops = model_flops_per_round(w)
     if flops and res["stage_ms"]["grad"] > 0:
@@ -532,6 +546,9 @@ def main():
                     help="also time the loop replayed from CUDA graphs of this many rounds (must divide --steps)")
     ap.add_argument("--mix-panel", type=int, default=None,
                     help="expert knob passed to dbw_set_mix_panel (1 = staged kernel, 2 = tensor-core kernel, 16..128 = panel width)")
+    ap.add_argument("--shard", default="none", choices=["none", "columns"],
+                    help="columns: ONE mix-only simulation split over the ranks by columns of X (no exchange; selection "
+                         "replicated; strong scaling) instead of one replica per rank")
     ap.add_argument("--samples", type=int, default=0, help="profiling aid: samples per worker instead of the config's")
     ap.add_argument("--width", type=int, default=0, help="profiling aid: columns d of the mix-only config instead of 2^20")
     args = ap.parse_args()

@@ -60,6 +60,8 @@ enum {
                                      does not hold deg_i - b_i entries for some i */
 #define DBW_STATUS_NAN_TIME 2u    /* some arrival time was NaN (ordered last) */
 #define DBW_STATUS_WAIT_TIMEOUT 4u /* a bounded pipeline wait expired; results of that call are invalid */
+#define DBW_STATUS_BOUNDS 32u     /* bounds-checked build only (libdbw_dbg.so): an index a kernel read from its own data
+                                     (graph, mixing plan, worker order) was out of range; the access was redirected */
 #define DBW_STATUS_INTERNAL 16u   /* a kernel found its own precomputed data inconsistent (should not happen) */
 #define DBW_STATUS_BAD_INDEX 8u   /* a batch index was outside [0, S) or a label outside [0, classes) (clamped) */
 

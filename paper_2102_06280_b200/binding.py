@@ -16,7 +16,7 @@ import numpy as np
 WEIGHT_METROPOLIS, WEIGHT_UNIFORM = 0, 1
 ORDER_LOCAL_THEN_MIX, ORDER_MIX_THEN_CORRECT = 0, 2
 GEMM_FP32, GEMM_BF16 = 0, 4
-STATUS_BAD_B, STATUS_NAN_TIME, STATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX, STATUS_INTERNAL = 1, 2, 4, 8, 16
+STATUS_BAD_B, STATUS_NAN_TIME, STATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX, STATUS_INTERNAL, STATUS_BOUNDS = 1, 2, 4, 8, 16, 32
 MAX_LAYERS = 8
 
 _ERR = {-1: "DBW_ERR_NULL", -2: "DBW_ERR_BAD_GRAPH", -3: "DBW_ERR_BAD_SHAPE", -4: "DBW_ERR_BAD_B",
@@ -38,7 +38,9 @@ class _ModelDesc(C.Structure):
                 ("w_off", C.c_int64 * MAX_LAYERS), ("b_off", C.c_int64 * MAX_LAYERS), ("batch", C.c_int32)]
 
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdbw.so")
+# DBW_LIBRARY=debug selects the bounds-checked build (libdbw_dbg.so, see build.py)
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         "libdbw_dbg.so" if os.environ.get("DBW_LIBRARY", "") == "debug" else "libdbw.so")
 _lib = None
 
 _P = C.c_void_p

@@ -220,6 +220,7 @@ int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* 
     h->smem_optin = (int)prop.sharedMemPerBlockOptin;
 
     h->plan.stride = std::max(4, (h->maxdeg + 3) / 4 * 4);
+    h->plan.n = N;
     const int D = N - 1;
     if ((rc = dev_alloc(&h->d_rowptr, N + 1)) || (rc = dev_alloc(&h->d_col, h->nnz)) ||
         (rc = dev_alloc(&h->d_links, 2 * D)) || (rc = dev_alloc(&h->d_covered, D)) ||
@@ -238,6 +239,7 @@ int dbw_init(dbw_handle** out, int32_t N, int64_t d, int64_t ld, const int32_t* 
               cuda_ok(cudaMemset(h->d_waited, 0, (size_t)N * sizeof(uint32_t))) &&
               cuda_ok(cudaMemset(h->d_ticket, 0, sizeof(uint32_t)));
     if (!ok) return fail(DBW_ERR_CUDA);
+    h->plan.status = h->d_status;
     if (!cuda_ok(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking)) ||
         !cuda_ok(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) ||
         !cuda_ok(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)))

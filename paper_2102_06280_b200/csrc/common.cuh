@@ -60,7 +60,22 @@ struct MixPlan {
     float* w_self = nullptr; // [N]
     int* cnt = nullptr;      // [N]
     int stride = 0;
+    int n = 0;                   // N (0 in a default-constructed plan: nothing to check against)
+    uint32_t* status = nullptr;  // the handle's status word, for the index checks of the bounds-checked build
 };
+
+// Index check of the bounds-checked build (-DDBW_BOUNDS, libdbw_dbg.so): an index outside [0, limit) that a
+// kernel read from its own data sets DBW_STATUS_BOUNDS and is replaced by 0, so that the access which follows
+// stays inside its array (nothing traps).  The regular build compiles the check away.
+__device__ __forceinline__ int checked(int idx, int limit, uint32_t* status) {
+#ifdef DBW_BOUNDS
+    if (limit > 0 && (idx < 0 || idx >= limit)) {
+        if (status) atomicOr(status, DBW_STATUS_BOUNDS);
+        return 0;
+    }
+#endif
+    return idx;
+}
 
 struct BF16State;  // tensor-core gradient path (grad_bf16.cu)
 struct TcMixState;  // tensor-core mix (mix_tc.cu)

@@ -29,7 +29,7 @@ update_backups_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* 
     int best_pos = 0x7fffffff;
     for (int pos = tid; pos < D; pos += kThreads) {
         if (covered[pos]) continue;
-        const double est = fmax(time_or_inf(t[links[2 * pos]], status), time_or_inf(t[links[2 * pos + 1]], status));
+        const double est = fmax(time_or_inf(t[checked(links[2 * pos], N, status)], status), time_or_inf(t[checked(links[2 * pos + 1], N, status)], status));
         if (est < best || (est == best && pos < best_pos)) {
             best = est;
             best_pos = pos;
@@ -80,7 +80,7 @@ update_backups_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* 
         const int lo = rowptr[j], hi = rowptr[j + 1];
         int p = 0;
         if (time_or_inf(t[j], status) <= theta)
-            for (int e = lo; e < hi; ++e) p += time_or_inf(t[col[e]], status) <= theta;
+            for (int e = lo; e < hi; ++e) p += time_or_inf(t[checked(col[e], N, status)], status) <= theta;
         b_out[j] = (hi - lo) - p;
     }
 }

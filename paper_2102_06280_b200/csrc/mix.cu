@@ -58,13 +58,14 @@ mix_direct_kernel(int N, long long ld, const float* __restrict__ X, const float*
         const float* pw = plan.w + (size_t)i * plan.stride;
         int k = 0;
         for (; k + 4 <= cnt; k += 4) {  // four neighbour rows in flight, added in list order
-            const float4 v0 = stepped(pi[k]), v1 = stepped(pi[k + 1]), v2 = stepped(pi[k + 2]), v3 = stepped(pi[k + 3]);
+            const float4 v0 = stepped(checked(pi[k], N, plan.status)), v1 = stepped(checked(pi[k + 1], N, plan.status)),
+                         v2 = stepped(checked(pi[k + 2], N, plan.status)), v3 = stepped(checked(pi[k + 3], N, plan.status));
             acc = fma4(pw[k], v0, acc);
             acc = fma4(pw[k + 1], v1, acc);
             acc = fma4(pw[k + 2], v2, acc);
             acc = fma4(pw[k + 3], v3, acc);
         }
-        for (; k < cnt; ++k) acc = fma4(pw[k], stepped(pi[k]), acc);
+        for (; k < cnt; ++k) acc = fma4(pw[k], stepped(checked(pi[k], N, plan.status)), acc);
         if (G && mix_then_correct) acc = fma4(-(lr_pw ? lr_pw[i] : lr), ldg4(G + (size_t)i * ld + c), acc);
         *reinterpret_cast<float4*>(Xout + (size_t)i * ld + c) = acc;
         if (shadow) *reinterpret_cast<uint2*>(shadow + (size_t)i * ld + c) = pack_bf16x4_rn(acc.x, acc.y, acc.z, acc.w);

@@ -435,6 +435,7 @@ mix_sp_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
             for (int q = 0; q < 4; ++q) {
                 const int r = j0 + 4 * (q & 1) + 16 * (q >> 1);
                 rows[q] = __ldg(a.order + kb * kKB + r);
+                if (rows[q] >= 0) rows[q] = checked(rows[q], a.N, a.status);
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -498,8 +499,8 @@ build_sparse_selection_kernel(int N, int k_pad, MixPlan plan, const int32_t* __r
     __syncthreads();
     if (i < N) {
         const int cnt = plan.cnt[i];
-        for (int k = threadIdx.x; k < cnt; k += blockDim.x) mark[pos[plan.idx[(size_t)i * plan.stride + k]]] = 1;
-        if (threadIdx.x == 0) mark[pos[i]] = 1;
+        for (int k = threadIdx.x; k < cnt; k += blockDim.x) mark[checked(pos[checked(plan.idx[(size_t)i * plan.stride + k], N, status)], k_pad, status)] = 1;
+        if (threadIdx.x == 0) mark[checked(pos[i], k_pad, status)] = 1;
     }
     __syncthreads();
     for (int e = threadIdx.x; e < k_pad / 16; e += blockDim.x) {

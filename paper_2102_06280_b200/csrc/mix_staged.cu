@@ -108,11 +108,11 @@ __global__ void __launch_bounds__(kThreads, 1) mix_staged_kernel(StagedArgs a) {
         for (int h = 0; h < 4; ++h) {
             const int k = k0 + 2 * h;
             auto entry = [&](int kk) -> uint32_t {
-                if (!WEIGHTED) return kk < cnt ? (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + kk] : (uint32_t)N;
+                if (!WEIGHTED) return kk < cnt ? (uint32_t)checked(a.plan.idx[(size_t)i * a.plan.stride + kk], N, a.plan.status) : (uint32_t)N;
                 if (kk >= cnt) return (uint32_t)i | ((uint32_t)kZeroCode << 10);
                 // the plan's weight is 1 / (1 + m): recover m (exact for m <= 62) and keep it as the code
                 const int m = __float2int_rn(1.0f / a.plan.w[(size_t)i * a.plan.stride + kk]) - 1;
-                return (uint32_t)a.plan.idx[(size_t)i * a.plan.stride + kk] | ((uint32_t)min(max(m, 0), kZeroCode - 1) << 10);
+                return (uint32_t)checked(a.plan.idx[(size_t)i * a.plan.stride + kk], N, a.plan.status) | ((uint32_t)min(max(m, 0), kZeroCode - 1) << 10);
             };
             w[h] = entry(k) | (entry(k + 1) << 16);
         }

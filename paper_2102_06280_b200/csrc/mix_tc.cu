@@ -462,7 +462,7 @@ build_selection_kernel(int N, int k_pad, MixPlan plan, uint16_t* S) {
     if (i >= N) return;
     __syncthreads();
     const int cnt = plan.cnt[i];
-    for (int k = threadIdx.x; k < cnt; k += blockDim.x) S[(size_t)i * k_pad + plan.idx[(size_t)i * plan.stride + k]] = 0x3F80u;
+    for (int k = threadIdx.x; k < cnt; k += blockDim.x) S[(size_t)i * k_pad + checked(plan.idx[(size_t)i * plan.stride + k], N, plan.status)] = 0x3F80u;
     if (threadIdx.x == 0) S[(size_t)i * k_pad + i] = 0x3F80u;
 }
 

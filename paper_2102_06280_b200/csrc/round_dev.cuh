@@ -272,7 +272,7 @@ __device__ __forceinline__ void plan_append(const MixPlan& plan, int i, int lane
                                             int& running) {
     unsigned m = __ballot_sync(0xffffffffu, keep);
     if (keep) {
-        int pos = running + __popc(m & ((1u << lane) - 1u));
+        const int pos = checked(running + __popc(m & ((1u << lane) - 1u)), plan.stride, plan.status);
         plan.idx[(size_t)i * plan.stride + pos] = j;
         plan.w[(size_t)i * plan.stride + pos] = w;
     }
@@ -311,7 +311,7 @@ __device__ __forceinline__ void select_worker(int i, int lane, const int32_t* __
     for (int base = 0; base < deg; base += 32) {
         const int e = lo + base + lane;
         const bool valid = e < hi;
-        const int j = valid ? col[e] : 0x7fffffff;
+        const int j = valid ? checked(col[e], plan.n, status) : 0x7fffffff;
         // arrival of col[e]'s update at worker i: the sender's time, or the link's own time
         const double tj = valid ? order_time(t_edge ? t_edge[e] : t[j], status) : 0.0;
         int rank = 0;
@@ -426,8 +426,10 @@ __device__ __forceinline__ void mix_panel_body(int panel, float4* sm, int N, lon
         const int4* pi = reinterpret_cast<const int4*>(plan.idx + (size_t)i * plan.stride);
         const float4* pw = reinterpret_cast<const float4*>(plan.w + (size_t)i * plan.stride);
         for (int k = 0; k < cnt; k += 4) {
-            const int4 j = load_g<NC>(pi + (k >> 2));
+            int4 j = load_g<NC>(pi + (k >> 2));
             const float4 w = load_g<NC>(pw + (k >> 2));
+            j.x = checked(j.x, N, plan.status); j.y = checked(j.y, N, plan.status);
+            j.z = checked(j.z, N, plan.status); j.w = checked(j.w, N, plan.status);
             acc = fma4(w.x, sm[j.x * GS + q], acc);
             acc = fma4(w.y, sm[j.y * GS + q], acc);
             acc = fma4(w.z, sm[j.z * GS + q], acc);

@@ -69,7 +69,7 @@ plan_kernel(int N, const int32_t* __restrict__ rowptr, const int32_t* __restrict
     for (int base = 0; base < deg; base += 32) {
         const int e = lo + base + lane;
         const bool keep = e < hi && kept[e] != 0;
-        const int j = e < hi ? col[e] : 0;
+        const int j = e < hi ? checked(col[e], N, status) : 0;
         float w = 0.f;
         if (keep) {
             const int dj = rowptr[j + 1] - rowptr[j];
@@ -155,8 +155,10 @@ extern "C" int dbw_select_static(int32_t N, const int32_t* rowptr, const int32_t
     // the array keeps whatever the previous call left: ticket, status and flags must start at zero
     DBW_CUDA(cudaMemsetAsync(base, 0, dbw::kStaticFlagsOff + sizeof(uint32_t) * (size_t)N, s));
     const int blocks = (N + dbw::kWarpsPerBlock - 1) / dbw::kWarpsPerBlock;
+    dbw::MixPlan no_plan{};
+    no_plan.n = N;  // only the bounds-checked build looks at it: this entry point's CSR is not validated on the host
     dbw::select_kernel<<<blocks, dbw::kWarpsPerBlock * 32, 0, s>>>(N, rowptr, col, t, nullptr, b, kept, tnbr, T_nbr, T_worker,
-                                                                   T_round, waited, ticket, status, dbw::MixPlan{}, 0, 0);
+                                                                   T_round, waited, ticket, status, no_plan, 0, 0);
     DBW_LAUNCHED();
     if (status_out) DBW_CUDA(cudaMemcpyAsync(status_out, status, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
     return DBW_OK;

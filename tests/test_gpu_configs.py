@@ -295,6 +295,39 @@ def test_mix_only_workloads_reduced_width(config, kernel):
     h.close()
 
 
+@pytest.mark.parametrize("config,panel", [(4, 0), (4, 3), (7, 0), (8, 0)])
+def test_column_shards_give_the_bits_of_the_whole_matrix(config, panel):
+    """The mix is independent per column (Eqs. 4-5), which is what a column-sharded run on several GPUs rests on:
+    every shard, run through its own handle as an N x width matrix, reproduces the whole-matrix result bit for
+    bit (same selection, same weights, same order of additions per element), with nothing exchanged."""
+    import paper_2102_06280_b200 as p
+    from paper_2102_06280_b200.sharding import column_shards
+    w = wl.make_workload(config, d=3000 + 4 * 37)
+    n, d = w.N, w.d
+    flags = p.WEIGHT_UNIFORM if w.weight_rule == "uniform" else 0
+    X = wl.gaussian_rows(w.init_seed, range(n), d)
+    G = wl.gaussian_rows(wl.external_gradient_seed(w), range(n), d, scale=0.01)
+    t = dev(wl.arrival_times(w, 1)[0])
+    b = dev(wl.uniform_backups(w, 1)[0])
+    kept = torch.zeros(len(w.col), dtype=torch.uint8, device="cuda")
+
+    def run(c0, c1):
+        h = p.Dbw(w.rowptr, w.col, d=c1 - c0, flags=flags)
+        if panel:
+            h.set_mix_panel(panel)
+        out = torch.empty(n, c1 - c0, device="cuda")
+        h.round(dev(X[:, c0:c1]), t, b, w.lr, out, kept, G_ext=dev(G[:, c0:c1]))
+        torch.cuda.synchronize()
+        assert h.status() == 0
+        h.close()
+        return out.cpu().numpy()
+
+    whole = run(0, d)
+    for world in (2, 3):
+        glued = np.concatenate([run(c0, c1) for c0, c1 in column_shards(d, world)], axis=1)
+        assert np.array_equal(glued, whole)
+
+
 def test_round_host_matches_device_round():
     """dbw_round_host (per-round inputs in pinned host memory) == dbw_round."""
     w = wl.make_workload(0)
