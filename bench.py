@@ -252,39 +252,87 @@ class ClockSampler:
 # CPU oracle timing (baseline leg and the reference arm)
 # ------------------------------------------------------------------------------------------
 
-def oracle_sample_seconds(w, k: int = 0, budget_s: float = 12.0):
-    """Times the oracle on a bounded sample of round k; returns (estimated s per full round, description).
+def _one_thread():
+    """Context manager pinning the BLAS / OpenMP pools of this process to one thread (no-op without threadpoolctl)."""
+    try:
+        from threadpoolctl import threadpool_limits
+        return threadpool_limits(limits=1)
+    except Exception:
+        import contextlib
+        return contextlib.nullcontext()
 
-    Selection, times, weights (and the threshold rule) run whole.  Gradients run for a few
-    workers and scale by N / sampled.  The mix runs on all rows x a block of columns and scales
-    by d / sampled columns (the update is independent per column).
+
+def _mix_block_seconds(job):
+    """Worker of the all-core leg: the oracle's mix on all rows x one block of columns, one thread; returns seconds."""
+    rowptr, col, ws, we, lr, n, cols, seed = job
+    from oracle import dbw_oracle as orc
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((n, cols)).astype(np.float32)
+    G = (0.01 * rng.standard_normal((n, cols))).astype(np.float32)
+    with _one_thread():
+        t0 = time.perf_counter()
+        orc.mix_update(rowptr, col, X, G, ws, we, lr)
+        return time.perf_counter() - t0
+
+
+def _grad_block_seconds(job):
+    """Worker of the all-core leg: the oracle's gradient of a few workers, one thread; returns seconds."""
+    config, overrides, k, workers = job
+    from oracle import dbw_oracle as orc
+    w = wl.make_workload(config, **overrides)
+    means = wl.class_means(w)
+    idx = wl.batch_indices(w, k)
+    data = [(wl.worker_dataset(w, i, means), wl.init_params(w, i)) for i in workers]
+    with _one_thread():
+        t0 = time.perf_counter()
+        for i, ((f, l), x) in zip(workers, data):
+            orc.mlp_grad(x, w.layers, f[idx[i]], l[idx[i]])
+        return time.perf_counter() - t0
+
+
+def oracle_sample_seconds(w, k: int = 0, budget_s: float = 12.0, pool=None, procs: int = 1, config=None, overrides=None):
+    """Times the oracle, as it stands, on a bounded sample of round k; returns (estimated s per full round, description).
+
+    Selection, times, weights (and the threshold rule) run whole.  Gradients run for a few workers and scale
+    by N / sampled.  The mix runs on all rows x a block of columns and scales by d / sampled columns (the
+    update is independent per column).  The timed code runs on ONE thread (BLAS pools pinned to one).  With a
+    process pool (`pool`, `procs` processes started with spawn) the gradient workers and the mix's column blocks
+    are spread over the processes, one thread each, and the slowest process counts: the all-core figure.
     """
     from oracle import dbw_oracle as orc
     rng = np.random.default_rng(123)
     t = wl.arrival_times(w, max(k + 1, 2))[k]
-    t0 = time.perf_counter()
-    if w.backups == "dtur":
-        b, _ = orc.Dtur(w.rowptr, w.col).update_backups(t)
-    elif w.backups == "uniform":
-        b = wl.uniform_backups(w, k + 1)[k]
-    else:
-        b = wl.fixed_backups(w)
-    kept = orc.select_fastest(w.rowptr, w.col, t, b)
-    orc.round_times(w.rowptr, w.col, t, b, kept)
-    ws, we = orc.mixing_weights(w.rowptr, w.col, b, kept, w.weight_rule)
-    t_discrete = time.perf_counter() - t0
+    with _one_thread():
+        t0 = time.perf_counter()
+        if w.backups == "dtur":
+            b, _ = orc.Dtur(w.rowptr, w.col).update_backups(t)
+        elif w.backups == "uniform":
+            b = wl.uniform_backups(w, k + 1)[k]
+        else:
+            b = wl.fixed_backups(w)
+        kept = orc.select_fastest(w.rowptr, w.col, t, b)
+        orc.round_times(w.rowptr, w.col, t, b, kept)
+        ws, we = orc.mixing_weights(w.rowptr, w.col, b, kept, w.weight_rule)
+        t_discrete = time.perf_counter() - t0
     t_grad, n_grad = 0.0, 0
-    if w.layers is not None:
+    if w.layers is not None and pool is None:
         means = wl.class_means(w)
         idx = wl.batch_indices(w, k)
         while n_grad < w.N and t_grad < budget_s / 2:
             i = n_grad
             f, l = wl.worker_dataset(w, i, means)
             x = wl.init_params(w, i)
-            t0 = time.perf_counter()
-            orc.mlp_grad(x, w.layers, f[idx[i]], l[idx[i]])
-            t_grad += time.perf_counter() - t0
+            with _one_thread():
+                t0 = time.perf_counter()
+                orc.mlp_grad(x, w.layers, f[idx[i]], l[idx[i]])
+                t_grad += time.perf_counter() - t0
             n_grad += 1
+        t_grad_full = t_grad * w.N / n_grad
+    elif w.layers is not None:
+        per = max(1, min(w.N // procs, 2))
+        jobs = [(config, overrides or {}, k, list(range(p * per, min(w.N, (p + 1) * per)))) for p in range(procs) if p * per < w.N]
+        t_grad = max(pool.map(_grad_block_seconds, jobs))
+        n_grad = sum(len(j[3]) for j in jobs)
         t_grad_full = t_grad * w.N / n_grad
     else:
         t_grad_full = 0.0
@@ -292,28 +340,43 @@ def oracle_sample_seconds(w, k: int = 0, budget_s: float = 12.0):
     t_mix, t_mix_full = 0.0, 0.0
     while True:
         cols = min(cols, w.d)
-        X = rng.standard_normal((w.N, cols)).astype(np.float32)
-        G = (0.01 * rng.standard_normal((w.N, cols))).astype(np.float32)
-        t0 = time.perf_counter()
-        orc.mix_update(w.rowptr, w.col, X, G, ws, we, w.lr)
-        t_mix = time.perf_counter() - t0
-        t_mix_full = t_mix * w.d / cols
-        if cols == w.d or t_mix > budget_s / 4:
+        if pool is None:
+            X = rng.standard_normal((w.N, cols)).astype(np.float32)
+            G = (0.01 * rng.standard_normal((w.N, cols))).astype(np.float32)
+            with _one_thread():
+                t0 = time.perf_counter()
+                orc.mix_update(w.rowptr, w.col, X, G, ws, we, w.lr)
+                t_mix = time.perf_counter() - t0
+            done_cols = cols
+        else:
+            t_mix = max(pool.map(_mix_block_seconds, [(w.rowptr, w.col, ws, we, w.lr, w.N, cols, 1000 + p) for p in range(procs)]))
+            done_cols = cols * procs
+        t_mix_full = t_mix * w.d / min(done_cols, w.d)
+        if done_cols >= w.d or t_mix > budget_s / 4:
             break
         cols *= 4
-    desc = ("round %d: selection/times/weights%s whole (%.3fs); gradients of %d of %d workers (%.2fs, scaled); "
+    desc = ("round %d on %s: selection/times/weights%s whole (%.3fs); gradients of %d of %d workers (%.2fs, scaled); "
             "mix on all %d rows x %d of %d columns (%.2fs, scaled)" %
-            (k, "/threshold rule" if w.backups == "dtur" else "", t_discrete, n_grad, w.N, t_grad, w.N, cols, w.d, t_mix))
+            (k, "1 thread" if pool is None else "%d processes x 1 thread" % procs,
+             "/threshold rule" if w.backups == "dtur" else "", t_discrete, n_grad, w.N, t_grad, w.N, min(done_cols, w.d), w.d, t_mix))
     return t_discrete + t_grad_full + t_mix_full, desc
 
 
-def cpu_threads():
-    try:
-        from threadpoolctl import threadpool_info
-        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-        return int(n)
-    except Exception:
-        return os.cpu_count() or 1
+def cpu_baseline(w, config, overrides, budget_s):
+    """The oracle on this host: on one thread, and spread over all cores (processes started with spawn, since the
+    CUDA context of this process must not be forked)."""
+    import multiprocessing as mp
+    sec1, desc1 = oracle_sample_seconds(w, 0, budget_s=budget_s)
+    out = {"value": w.N / sec1, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc1}
+    procs = max(1, min(os.cpu_count() or 1, 64))
+    if procs > 1:
+        try:
+            with mp.get_context("spawn").Pool(procs) as pool:
+                secp, descp = oracle_sample_seconds(w, 0, budget_s=budget_s, pool=pool, procs=procs, config=config, overrides=overrides)
+            out["all_cores"] = {"value": w.N / secp, "unit": UNIT, "cores": procs, "sample": descp}
+        except Exception as e:  # a host that cannot start the pool still reports the one-thread figure
+            out["all_cores"] = {"error": repr(e)}
+    return out
 
 
 def run_reference(args):
@@ -336,7 +399,7 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "N": w.N, "d": w.d, "note": "CPU oracle, each step a bounded sample scaled to a full round"},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -431,8 +494,7 @@ def run_ours(args):
     if extra:
         line["other_workloads"] = extra
     if not args.no_cpu_baseline and world == 1:
-        sec, desc = oracle_sample_seconds(w, 0, budget_s=args.ref_budget)
-        line["cpu_baseline"] = {"value": w.N / sec, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc}
+        line["cpu_baseline"] = cpu_baseline(w, args.config, overrides, args.ref_budget)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -484,6 +546,24 @@ def model_flops_per_round(w):
     return per_sample * w.batch * w.N
 
 
+def tensor_core_gemm_work(w):
+    """(flops, bytes) of the tensor-core GEMM launches of one round: forward, dW and (above the first layer) dA of
+    every layer but the last.  Bytes = what each launch must move once: its two bf16 operands, its output (bf16
+    activations / dZ, fp32 dW into G), the fp32 bias or the bf16 ReLU mask."""
+    if w.layers is None or w.precision != "bf16":
+        return 0, 0
+    dims = wl.layer_dims(w.layers)          # [(out, in)] per layer
+    B, flops, nbytes = w.batch, 0, 0
+    for l, (o, i) in enumerate(dims[:-1]):
+        flops += 2 * B * i * o * 2                                   # forward, dW
+        nbytes += (B * i * 2 + i * o * 2 + B * o * 2 + o * 4)        # forward: A_l, W_l, A_{l+1}, bias
+        nbytes += (B * o * 2 + B * i * 2 + i * o * 4)                # dW: dZ_{l+1}, A_l, fp32 dW
+        if l >= 1:
+            flops += 2 * B * i * o                                   # dA
+            nbytes += (B * o * 2 + i * o * 2 + B * i * 2 + B * i * 2)  # dA: dZ_{l+1}, W_l, mask A_l, dZ_l
+    return flops * w.N, nbytes * w.N
+
+
 def summary(res, world, args):
     w = res["w"]
     peaks, peak_kind = measured_peaks()
@@ -528,6 +608,20 @@ def summary(res, world, args):
         out["gradients"] = {"dense_flop_per_round": flops,
                             "tflops_over_grad_stage": flops / (res["stage_ms"]["grad"] * 1e-3) / 1e12,
                             "note": "grad stage = gather, casts, GEMMs, loss and last layer together"}
+    tc_flops, tc_bytes = tensor_core_gemm_work(w)
+    gemm_ms = res["stage_ms"].get("gemm", 0.0)
+    if tc_flops and gemm_ms > 0:
+        # The dense layers' GEMMs (batch 128-256 per worker) stream their weights or their fp32 result once: they sit
+        # between the two rooflines, so both are reported: flops over the tensor peak a long step sustains, and
+        # the bytes each launch must move over the copy bandwidth.
+        tf = tc_flops / (gemm_ms * 1e-3) / 1e12
+        gbs = tc_bytes / (gemm_ms * 1e-3) / 1e9
+        peak_tf = peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops"))
+        out["roofline_gemm"] = {"kernel": "gemm_tc_kernel (all tensor-core launches of a round)", "ms_per_round": gemm_ms,
+                                "flop_per_round": tc_flops, "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+                                "frac": tf / peak_tf, "peak_kind": "sustained bf16, of " + peak_kind,
+                                "hbm_bytes_per_round": tc_bytes, "achieved_gbs": gbs, "frac_hbm": gbs / peaks["hbm_gbs"],
+                                "bound": "hbm" if gbs / peaks["hbm_gbs"] > tf / peak_tf else "tensor"}
     return out
 
 

@@ -287,7 +287,8 @@ int dbw_get_links(const dbw_handle* h, int32_t* links);
  * gradients the selection, which needs only t and b, runs beside them on a stream of the handle
  * (forked from and joined back into the caller's stream), so the three times may add up to more
  * than the round took.  dbw_profile_read() waits for the recorded events, adds their elapsed times to
- * ms[3] (HOST), stores the number of rounds in *rounds and clears the record.  Do not enable
+ * ms[4] (HOST: the three stages, then ms[3] = the tensor-core GEMM launches inside the gradient stage, each
+ * between events of its own; 0 on the fp32 path), stores the number of rounds in *rounds and clears the record.  Do not enable
  * it while the stream is being captured into a CUDA graph.
  */
 int dbw_profile(dbw_handle* h, int enable);

@@ -264,11 +264,12 @@ class Dbw:
         _check(lib().dbw_profile(self._h, int(bool(enable))), "dbw_profile")
 
     def profile_read(self):
-        """({'grad': ms, 'select': ms, 'mix': ms}, rounds) accumulated since the last read."""
-        ms = (C.c_double * 3)(0.0, 0.0, 0.0)
+        """({'grad': ms, 'select': ms, 'mix': ms, 'gemm': ms}, rounds) accumulated since the last read
+        ('gemm' = the tensor-core GEMM launches inside the gradient stage)."""
+        ms = (C.c_double * 4)(0.0, 0.0, 0.0, 0.0)
         n = C.c_int32(0)
         _check(lib().dbw_profile_read(self._h, ms, C.byref(n)), "dbw_profile_read")
-        return {"grad": ms[0], "select": ms[1], "mix": ms[2]}, int(n.value)
+        return {"grad": ms[0], "select": ms[1], "mix": ms[2], "gemm": ms[3]}, int(n.value)
 
     def debug_wait_probe(self, polls: int, out):
         _check(lib().dbw_debug_wait_probe(self._h, int(polls), _ptr(out), _stream()), "dbw_debug_wait_probe")

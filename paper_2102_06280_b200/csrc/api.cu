@@ -111,7 +111,9 @@ int dev_alloc(T** p, size_t n) {
 
 void free_all(dbw_handle* h) {
     for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->prof_gemm_events) cudaEventDestroy(e);
     h->prof_events.clear();
+    h->prof_gemm_events.clear();
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->side) cudaStreamDestroy(h->side);
@@ -419,6 +421,7 @@ int dbw_round(dbw_handle* h, const float* X, const double* t, const int32_t* b, 
 int dbw_profile(dbw_handle* h, int enable) {
     if (!h) return DBW_ERR_NULL;
     h->profiling = enable != 0;
+    if (!h->profiling) h->prof_gemm_used = 0;
     return DBW_OK;
 }
 
@@ -441,6 +444,13 @@ int dbw_profile_read(dbw_handle* h, double* ms, int32_t* rounds) {
             ms[st] += v;
         }
     }
+    for (int e = 0; e + 1 < h->prof_gemm_used; e += 2) {  // the tensor-core GEMM launches of those rounds
+        float v = 0.f;
+        DBW_CUDA(cudaEventSynchronize(h->prof_gemm_events[e + 1]));
+        DBW_CUDA(cudaEventElapsedTime(&v, h->prof_gemm_events[e], h->prof_gemm_events[e + 1]));
+        ms[3] += v;
+    }
+    h->prof_gemm_used = 0;
     *rounds = h->prof_rounds;
     h->prof_rounds = 0;
     return DBW_OK;

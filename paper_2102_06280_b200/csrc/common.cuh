@@ -145,6 +145,8 @@ struct dbw_handle {
     // stage timing (dbw_profile): events[round][0..5] = start / end of the gradient, selection and mix stages
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;
+    std::vector<cudaEvent_t> prof_gemm_events;  // pairs around every tensor-core GEMM launch while profiling
+    int prof_gemm_used = 0;
     std::vector<char> prof_single;  // per recorded round: 1 = single-launch round (events 0 and 1 only)
     int prof_rounds = 0;
 
