@@ -608,7 +608,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // in v[0] and v[1].  Each step halves what a lane keeps and hands the other half to the lane it pairs with.
 __device__ __forceinline__ void lane_sum64(float (&v)[64], int lane) {
 #pragma unroll
-    for (int half = 32, mask = 16; half >= 1; half >>= 1, mask >>= 1) {
+    for (int half = 32, mask = 16; half >= 2; half >>= 1, mask >>= 1) {
         const bool upper = (lane & mask) != 0;
 #pragma unroll
         for (int i = 0; i < half; ++i) {
