@@ -580,231 +580,6 @@ head_reduce_kernel(int B, int K, int C, int parts, int workers, const float* __r
     }
 }
 
-// ----------------------------------------------------------------------------- last layer, fused
-// Forward (logits from the fp32 master weights), softmax cross-entropy, loss, and the whole backward of
-// the last layer in ONE kernel that reads every row of A_{L-1} from global memory once:
-//   logits[s][c] = A[s,:] . W[c,:] + b[c];  dZ[s][c] = (softmax - onehot) / B;  loss = mean(lse - z_y)
-//   dW[c][k] = sum_s dZ[s][c] A[s][k];  db[c] = sum_s dZ[s][c];
-//   dZprev[s][k] = [A[s][k] > 0] * sum_c dZ[s][c] W[c][k]                     (bf16)
-// A block owns one worker (or one of `parts` slices of its batch) and walks the samples in chunks of 32
-// that are staged in shared memory (next chunk in flight by cp.async while this one is used).
-//   logits: a warp takes four samples and one K range; each lane owns eight consecutive k of every 256
-//     (128-bit shared loads of A and W), 4 x 16 partial sums per lane, summed over the lanes by a halving
-//     exchange (62 shuffles instead of 320), K ranges added in a fixed order through shared memory;
-//   backward: a thread owns two consecutive k for the whole batch: W[c][k], dW[c][k] live in registers,
-//     dZ of the chunk is read as 128-bit broadcasts, dZprev leaves as coalesced bf16 pairs.
-// Sums over the batch run in sample order, the loss reduction is the one of loss_reduce_kernel.
-constexpr int HF_CHUNK = 32;   // samples per chunk
-constexpr int HF_CP = 16;      // class slots of the logits stage and of the dZ rows in shared memory
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// Sum of v[slot] over the 32 lanes for 64 slots: afterwards lane l holds the totals of slots 2l and 2l+1
-// in v[0] and v[1].  Each step halves what a lane keeps and hands the other half to the lane it pairs with.
-__device__ __forceinline__ void lane_sum64(float (&v)[64], int lane) {
-#pragma unroll
-    for (int half = 32, mask = 16; half >= 2; half >>= 1, mask >>= 1) {
-        const bool upper = (lane & mask) != 0;
-#pragma unroll
-        for (int i = 0; i < half; ++i) {
-            const float keep = upper ? v[i + half] : v[i];
-            const float send = upper ? v[i] : v[i + half];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
-        }
-    }
-}
-
-struct HeadArgs {
-    int B, K, C, parts;
-    const bf16* A;      // [N][B][K]
-    const float* X;     // master parameters, row pitch ld
-    long long ld, w_off, b_off;
-    const int32_t* ylab;
-    float* G;           // dW, db of the last layer (parts == 1)
-    float* dwp;         // [parts][N][C][K] partial dW (parts > 1)
-    float* dzL;         // [N][B][C] (written when parts > 1: head_reduce_kernel sums db from it)
-    float* loss_s;      // [N][B]   (written when parts > 1)
-    float* loss;        // [N] nullable (parts == 1)
-    bf16* dzP;          // [N][B][K] nullable
-};
-
-// CB = class slots of the backward stage (10 for up to ten classes, else 16).
-template <int CB>
-__global__ void __launch_bounds__(512, 1) head_fused_kernel(HeadArgs a) {
-    extern __shared__ __align__(16) uint8_t hsm[];
-    const int K = a.K, C = a.C, B = a.B;
-    const int wpitch = K + 4;                                    // fp32 row pitch of W in shared memory (bank spread)
-    float* sW = reinterpret_cast<float*>(hsm);                   // [HF_CP][wpitch]
-    bf16* sA = reinterpret_cast<bf16*>(sW + HF_CP * wpitch);     // [2][HF_CHUNK][K]
-    float* sdz = reinterpret_cast<float*>(sA + 2 * HF_CHUNK * K);  // [HF_CHUNK][HF_CP]
-    float* slog = sdz + HF_CHUNK * HF_CP;                        // [2][HF_CHUNK][HF_CP] partial logits of the K ranges
-    float* sloss = slog + 2 * HF_CHUNK * HF_CP;                  // [B] per-sample losses of this block's samples
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    const int i = blockIdx.y, part = blockIdx.x;
-    const int nch = B / 8;
-    const int s_lo = 8 * (int)((long long)part * nch / a.parts), s_hi = 8 * (int)((long long)(part + 1) * nch / a.parts);
-    const float* Wg = a.X + (size_t)i * a.ld + a.w_off;
-    const bf16* Ag = a.A + (size_t)i * B * K;
-
-    auto stage = [&](int s0, int buf) {  // samples s0 .. s0+31 (those below s_hi) -> sA[buf]
-        const int segs = K / 8;           // 16-byte segments per sample
-        for (int e = tid; e < HF_CHUNK * segs; e += blockDim.x) {
-            const int s = e / segs, g = e % segs;
-            if (s0 + s < s_hi) cp_async16(sA + ((size_t)buf * HF_CHUNK + s) * K + g * 8, Ag + (size_t)(s0 + s) * K + g * 8);
-        }
-        cp_async_commit();
-    };
-    stage(s_lo, 0);
-    for (int e = tid; e < HF_CP * (K / 4); e += blockDim.x) {     // W (zero rows above C)
-        const int c = e / (K / 4), k4 = e % (K / 4);
-        const float4 v = c < C ? __ldg(reinterpret_cast<const float4*>(Wg + (size_t)c * K) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        *reinterpret_cast<float4*>(sW + (size_t)c * wpitch + 4 * k4) = v;
-    }
-    // backward stage: this thread's two k
-    const int k = 2 * tid;
-    const bool k_ok = k < K;
-    float dw[CB][2];
-#pragma unroll
-    for (int c = 0; c < CB; ++c) dw[c][0] = dw[c][1] = 0.f;
-    float db = 0.f;                                               // thread c < C: sum of dZ[s][c] in sample order
-    const float invB = 1.0f / (float)B;
-    const int n_ranges = nwarps >= 16 ? 2 : 1;                    // K ranges of the logits stage
-    const int k_range = (K / n_ranges + 7) / 8 * 8;
-
-    int buf = 0;
-    for (int s0 = s_lo; s0 < s_hi; s0 += HF_CHUNK, buf ^= 1) {
-        if (s0 + HF_CHUNK < s_hi) {
-            stage(s0 + HF_CHUNK, buf ^ 1);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();                                          // chunk (and, the first time, W) visible to all
-        const bf16* cA = sA + (size_t)buf * HF_CHUNK * K;
-        const int n_s = min(HF_CHUNK, s_hi - s0);
-        // ---- logits: tasks = 8 sample groups x K ranges ----
-        for (int task = warp; task < 8 * n_ranges; task += nwarps) {
-            const int g4 = task % 8, range = task / 8;
-            float acc[64];
-#pragma unroll
-            for (int e = 0; e < 64; ++e) acc[e] = 0.f;
-            const int k_end = min(K, (range + 1) * k_range);
-            for (int kk = range * k_range + lane * 8; kk < k_end; kk += 256) {
-                uint32_t raw[4][4];  // eight bf16 of four samples; bf16 -> fp32 is a 16-bit shift, done at the use
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint4 r = *reinterpret_cast<const uint4*>(cA + (size_t)(4 * g4 + u) * K + kk);
-                    raw[u][0] = r.x; raw[u][1] = r.y; raw[u][2] = r.z; raw[u][3] = r.w;
-                }
-#pragma unroll
-                for (int c = 0; c < HF_CP; ++c) {
-                    const float4 w0 = *reinterpret_cast<const float4*>(sW + (size_t)c * wpitch + kk);
-                    const float4 w1 = *reinterpret_cast<const float4*>(sW + (size_t)c * wpitch + kk + 4);
-                    const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            acc[u * HF_CP + c] = fmaf(__uint_as_float(raw[u][e] << 16), wv[2 * e], acc[u * HF_CP + c]);
-                            acc[u * HF_CP + c] = fmaf(__uint_as_float(raw[u][e] & 0xffff0000u), wv[2 * e + 1], acc[u * HF_CP + c]);
-                        }
-                }
-            }
-            lane_sum64(acc, lane);                                // lane l: slots 2l, 2l+1 = sample l/8, classes 2(l%8), +1
-            float* dst = slog + ((size_t)range * HF_CHUNK + 4 * g4 + (lane >> 3)) * HF_CP + 2 * (lane & 7);
-            dst[0] = acc[0];
-            dst[1] = acc[1];
-        }
-        __syncthreads();
-        // ---- softmax, dZ, per-sample loss: a warp per sample, lane = class ----
-        for (int s = warp; s < n_s; s += nwarps) {
-            float z = -INFINITY;
-            if (lane < C) {
-                z = slog[(size_t)s * HF_CP + lane];
-                if (n_ranges == 2) z += slog[((size_t)HF_CHUNK + s) * HF_CP + lane];
-                z += a.X[(size_t)i * a.ld + a.b_off + lane];
-            }
-            float mx = z;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            const float e = lane < C ? expf(z - mx) : 0.f;
-            float sum = e;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            const int y = a.ylab[(size_t)i * B + s0 + s];
-            const float d = lane < C ? (e / sum - (lane == y ? 1.f : 0.f)) * invB : 0.f;
-            if (lane < HF_CP) sdz[(size_t)s * HF_CP + lane] = d;
-            if (a.parts > 1 && lane < C) a.dzL[((size_t)i * B + s0 + s) * C + lane] = d;
-            const float zy = __shfl_sync(0xffffffffu, z, y & 31);
-            if (lane == 0) sloss[s0 - s_lo + s] = (mx + logf(sum)) - zy;
-        }
-        __syncthreads();
-        // ---- backward of the chunk ----
-        if (tid < C)
-            for (int s = 0; s < n_s; ++s) db += sdz[(size_t)s * HF_CP + tid];
-        if (k_ok) {
-            float w[CB][2];                                       // this thread's two columns of W (rows above C are zero)
-#pragma unroll
-            for (int c = 0; c < CB; ++c) {
-                const float2 w2 = *reinterpret_cast<const float2*>(sW + (size_t)c * wpitch + k);
-                w[c][0] = w2.x;
-                w[c][1] = w2.y;
-            }
-            for (int s = 0; s < n_s; ++s) {
-                const uint32_t raw = *reinterpret_cast<const uint32_t*>(cA + (size_t)s * K + k);
-                const float a0 = __uint_as_float(raw << 16), a1 = __uint_as_float(raw & 0xffff0000u);
-                float da0 = 0.f, da1 = 0.f;
-#pragma unroll
-                for (int c4 = 0; c4 < (CB + 3) / 4; ++c4) {
-                    const float4 d4 = *reinterpret_cast<const float4*>(sdz + (size_t)s * HF_CP + 4 * c4);
-                    const float dz[4] = {d4.x, d4.y, d4.z, d4.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int c = 4 * c4 + e;
-                        if (c < CB) {
-                            dw[c][0] = fmaf(dz[e], a0, dw[c][0]);
-                            dw[c][1] = fmaf(dz[e], a1, dw[c][1]);
-                            da0 = fmaf(dz[e], w[c][0], da0);
-                            da1 = fmaf(dz[e], w[c][1], da1);
-                        }
-                    }
-                }
-                if (a.dzP)
-                    *reinterpret_cast<uint32_t*>(a.dzP + ((size_t)i * B + s0 + s) * K + k) = pack_bf16x2(a0 > 0.f ? da0 : 0.f, a1 > 0.f ? da1 : 0.f);
-            }
-        }
-        __syncthreads();                                          // the chunk buffer and sdz are free again
-    }
-    // ---- results ----
-    if (k_ok) {
-        float* dst = a.parts == 1 ? a.G + (size_t)i * a.ld + a.w_off : a.dwp + ((size_t)part * gridDim.y + i) * C * K;
-#pragma unroll
-        for (int c = 0; c < CB; ++c)
-            if (c < C) *reinterpret_cast<float2*>(dst + (size_t)c * K + k) = make_float2(dw[c][0], dw[c][1]);
-    }
-    if (a.parts == 1) {
-        if (tid < C) a.G[(size_t)i * a.ld + a.b_off + tid] = db;
-        if (warp == 0 && a.loss) {                                // the reduction of loss_reduce_kernel
-            float t = 0.f;
-            for (int m = lane; m < B; m += 32) t += sloss[m];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-            if (lane == 0) a.loss[i] = t / (float)B;
-        }
-    } else {
-        for (int m = tid; m < s_hi - s_lo; m += blockDim.x) a.loss_s[(size_t)i * B + s_lo + m] = sloss[m];
-    }
-}
-
-size_t head_fused_smem(int K, int B) {
-    return (size_t)HF_CP * (K + 4) * 4 + (size_t)2 * HF_CHUNK * K * 2 + (size_t)HF_CHUNK * HF_CP * 4 * 3 + (size_t)B * 4;
-}
-
 // ----------------------------------------------------------------------------- host side
 // MN-major operand [workers][K rows][MN] bf16 (MN contiguous): box = 64 (MN) x 64 (K rows) x 1.
 bool make_operand_map_mn(CUtensorMap* map, const bf16* base, int MN, int Krows, int workers, long long worker_pitch = 0) {
@@ -848,7 +623,6 @@ struct BF16State {
     int32_t* ylab = nullptr;         // [N][B]
     CUtensorMap fwdA[DBW_MAX_LAYERS], fwdB[DBW_MAX_LAYERS], dwA[DBW_MAX_LAYERS], dwB[DBW_MAX_LAYERS],
         daA[DBW_MAX_LAYERS], daB[DBW_MAX_LAYERS];
-    bool head_fused = false;         // the last layer runs as one kernel (head_fused_kernel)
     std::vector<void*> owned;
 };
 
@@ -955,13 +729,6 @@ int grad_bf16_alloc(dbw_handle* h) {
         }
     }
     if (!ok) return DBW_ERR_CUDA;
-    // the fused last-layer kernel: up to 16 classes, a thread per two input features, its staging within shared memory
-    const int K_last = m.dims[L - 1];
-    if (m.dims[L] <= HF_CP && K_last <= 1024 && B % 8 == 0 && head_fused_smem(K_last, B) <= (size_t)h->smem_optin) {
-        DBW_CUDA(cudaFuncSetAttribute(head_fused_kernel<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_fused_smem(K_last, B)));
-        DBW_CUDA(cudaFuncSetAttribute(head_fused_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_fused_smem(K_last, B)));
-        st->head_fused = true;
-    }
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -1009,57 +776,31 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
-    if (st->head_fused) {
-        // one kernel that reads A_{L-1} once; the batch is split over blocks only when the workers alone leave SMs idle
-        int parts = 1;
-        if (4 * N < 3 * h->sm_count) parts = std::max(1, std::min(std::min(4, h->sm_count / N), B / (2 * HF_CHUNK)));
-        HeadArgs a{};
-        a.B = B; a.K = K; a.C = C; a.parts = parts;
-        a.A = st->A[L - 1]; a.X = X; a.ld = h->ld; a.w_off = m.w_off[L - 1]; a.b_off = m.b_off[L - 1];
-        a.ylab = st->ylab; a.G = G; a.dwp = st->dwp; a.dzL = st->dzL; a.loss_s = st->loss_s; a.loss = loss; a.dzP = dzP;
-        const int threads = std::max(32, (K / 2 + 31) / 32 * 32);
-        const size_t smem = head_fused_smem(K, B);
-        if (C <= 10)
-            head_fused_kernel<10><<<dim3(parts, N), threads, smem, s>>>(a);
-        else
-            head_fused_kernel<16><<<dim3(parts, N), threads, smem, s>>>(a);
-        DBW_LAUNCHED();
-        if (parts > 1) {
-            if (loss) {
-                loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
-                DBW_LAUNCHED();
-            }
-            head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
-                                                                                      m.w_off[L - 1], m.b_off[L - 1]);
-            DBW_LAUNCHED();
-        }
-    } else {
-        if (C <= 16)
-            head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
-                                                                           m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
-        else
-            head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
-                                                                           m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
-        DBW_LAUNCHED();
-        if (loss) {
-            loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
-            DBW_LAUNCHED();
-        }
-        const int parts = B >= 64 ? 4 : 1;
-        if (C <= 12)  // ten classes: a quarter fewer multiply-adds than with the 16-class instance
-            head_backward_kernel<12, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 12 * 4, s>>>(
-                B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
-        else if (C <= 16)
-            head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
-                B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
-        else
-            head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N, parts), 64, (size_t)B * 32 * 4, s>>>(
-                B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
-        DBW_LAUNCHED();
-        head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
-                                                                                  m.w_off[L - 1], m.b_off[L - 1]);
+    if (C <= 16)
+        head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+                                                                       m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
+    else
+        head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
+                                                                       m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
+    DBW_LAUNCHED();
+    if (loss) {
+        loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
         DBW_LAUNCHED();
     }
+    const int parts = B >= 64 ? 4 : 1;
+    if (C <= 12)  // ten classes: a quarter fewer multiply-adds than with the 16-class instance
+        head_backward_kernel<12, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 12 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
+    else if (C <= 16)
+        head_backward_kernel<16, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 16 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
+    else
+        head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N, parts), 64, (size_t)B * 32 * 4, s>>>(
+            B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
+    DBW_LAUNCHED();
+    head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
+                                                                              m.w_off[L - 1], m.b_off[L - 1]);
+    DBW_LAUNCHED();
     // backward through the tensor-core layers
     for (int l = L - 2; l >= 0; --l) {
         const int in = m.dims[l], out = m.dims[l + 1];
