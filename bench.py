@@ -33,10 +33,13 @@ from workloads import configs as wl  # noqa: E402
 METRIC = "simulated worker-rounds/sec"
 UNIT = "worker-rounds/s"
 DEFAULT_CONFIG = 4
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix kernel, from the ncu captures
-# summarised under profiles/ (small case scaled by the columns processed); None = not captured for
-# this workload or the kernel changed since.
-MIX_TRAFFIC_BYTES = {4: (537.1e6 + 220.4e6) * 16}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix kernel, from the ncu captures summarised
+# under profiles/ (config 4: the d = 65,536 case scaled by 16, the traffic being proportional to the columns
+# processed; configs 2 and 3: their mix at full size).  Reported only for the kernel the capture was taken of;
+# None = not captured for this workload.
+MIX_TRAFFIC_BYTES = {4: ("mix_staged_kernel", (537.05e6 + 220.89e6) * 16),
+                     3: ("mix_panel_kernel", 4.316048e9 + 3.227908e9),
+                     2: ("mix_panel_kernel", 875.2448e6 + 612.1979e6)}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -55,7 +58,7 @@ def measured_peaks():
 class Job:
     """One workload resident on one GPU, stepped through the C ABI."""
 
-    def __init__(self, config: int, device: int = 0, rounds: int | None = None, col_range=None, **overrides):
+    def __init__(self, config: int, device: int = 0, rounds: int | None = None, col_range=None, consensus_only=False, **overrides):
         """col_range = (c0, c1): this job owns only those columns of a mix-only workload's matrices (one column
         shard of several; the update is independent per column, see paper_2102_06280_b200/sharding.py)."""
         import torch
@@ -99,6 +102,9 @@ class Job:
                 self.G[r0:r0 + step].copy_(torch.from_numpy(np.ascontiguousarray(
                     wl.gaussian_rows(wl.external_gradient_seed(w), rows, w.d, scale=0.01)[:, c0:c1])))
             self.h_idx = self.d_idx = None
+            if consensus_only:      # the truncated model's tail (Section 3.2.1): G = 0, no gradient matrix is read
+                self.G = None
+        self.consensus_only = consensus_only and w.layers is None
         self.h_t = torch.from_numpy(wl.arrival_times(w, self.n_rounds)).pin_memory()
         self.d_t = self.h_t.to(self.dev)
         if w.backups == "fixed":
@@ -190,7 +196,7 @@ class Job:
         return h2d, d2h
 
     def mix_bytes_per_launch(self):
-        return 12 * self.w.N * self.ld
+        return (8 if self.consensus_only else 12) * self.w.N * self.ld
 
     def close(self):
         self.h.close()
@@ -488,8 +494,10 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "strong" if args.shard == "columns" else "weak", "vs_baseline": None,
             "data": "synthetic"}
     line.update(summary(res, world, args))
-    line["roofline"]["traffic"] = (MIX_TRAFFIC_BYTES.get(args.config)
-                                   if not overrides and res["mix_kernel"] == "mix_staged_kernel" else None)
+    if overrides or col_range is not None or args.consensus_only:
+        line["roofline"]["traffic"] = None
+    if args.consensus_only:
+        line["config"]["gradients"] = "none (consensus-only iterations: 8 B per element)"
     line["clocks"] = clocks
     if extra:
         line["other_workloads"] = extra
@@ -504,7 +512,7 @@ def measure(config, local, args, dist, overrides, col_range=None):
     """Device-resident loop, stage times, launch count and the end-to-end loop of one workload."""
     import torch
     from paper_2102_06280_b200 import binding
-    job = Job(config, device=local, col_range=col_range, **overrides)
+    job = Job(config, device=local, col_range=col_range, consensus_only=getattr(args, "consensus_only", False), **overrides)
     if args.mix_panel is not None:
         job.h.set_mix_panel(args.mix_panel)
     for _ in range(args.warmup):
@@ -586,7 +594,9 @@ def summary(res, world, args):
            "gpu_launches": int(res["launches"]),
            "roofline": {"kernel": res["mix_kernel"], "bound": "hbm",
                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
+                        "peak_kind": "of " + peak_kind, "frac_of_8TBps_nominal": achieved / 8000.0,
+                        "traffic": (MIX_TRAFFIC_BYTES[w.index][1] if w.index in MIX_TRAFFIC_BYTES and
+                                    MIX_TRAFFIC_BYTES[w.index][0] == res["mix_kernel"] else None),
                         "bytes_per_launch": res["mix_bytes"], "ms_per_launch": mix_ms},
            "device_status": res["status"]}
     # The second roofline of the mix: every output element needs (1 + kept neighbours) fp32 operands out
@@ -640,6 +650,8 @@ def main():
                     help="also time the loop replayed from CUDA graphs of this many rounds (must divide --steps)")
     ap.add_argument("--mix-panel", type=int, default=None,
                     help="expert knob passed to dbw_set_mix_panel (1 = staged kernel, 2 = tensor-core kernel, 16..128 = panel width)")
+    ap.add_argument("--consensus-only", action="store_true",
+                    help="mix-only workloads: consensus-only iterations (G = 0, nothing of G read): 8 bytes per element")
     ap.add_argument("--shard", default="none", choices=["none", "columns"],
                     help="columns: ONE mix-only simulation split over the ranks by columns of X (no exchange; selection "
                          "replicated; strong scaling) instead of one replica per rank")
