@@ -213,6 +213,16 @@ int launch_round_fused(dbw_handle* h, const float* X, const double* t, const int
 int launch_update_backups(dbw_handle* h, const double* t, int32_t* b_out, double* theta_out, cudaStream_t s);
 
 // grad_fp32.cu
+// fp32 gradient path: shared memory of the last layer's backward step (the worker's dZ and its row offsets),
+// and whether the last layer can take the small-output path (at most 32 classes, 16-byte rows).
+inline size_t fp32_head_smem_bytes(int B, int C) { return (size_t)((B * C + 1) & ~1) * 4 + (size_t)B * 8; }
+inline bool fp32_head_usable(const dbw_handle* h) {
+    const dbw_model_desc& m = h->model;
+    const int L = m.n_layers;
+    if (L < 1) return false;
+    return m.dims[L] <= 32 && (m.dims[L - 1] & 3) == 0 && (m.w_off[L - 1] & 3) == 0 && (h->ld & 3) == 0 &&
+           ((uintptr_t)h->feat & 15) == 0 && fp32_head_smem_bytes(m.batch, m.dims[L]) <= 32768;
+}
 int grad_fp32_alloc(dbw_handle* h);
 void grad_fp32_free(dbw_handle* h);
 int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, float* G, float* loss,

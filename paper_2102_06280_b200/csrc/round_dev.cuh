@@ -235,6 +235,197 @@ __device__ __forceinline__ void bias_grad_col(int i, int o, int B, int out_dim, 
 }
 
 
+// ------------------------------------------------------------------ last layer with at most 32 classes (Eq. 2)
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// A layer with a handful of outputs is a poor GEMM (one 32-wide tile, mostly padding, and a reduction as
+// long as the layer is wide), so the last layer's forward pass, the loss and its backward pass run as two
+// steps of their own: a warp per sample forward (every lane a slice of the features, all classes at once),
+// and eight lanes per four features backward (the worker's dZ out of shared memory).
+// For a one-layer model the rows are read straight from the data set through the batch indices.
+struct HeadRows {
+    const float* act;            // [N][B][in] output of the layer before, or null
+    const int32_t* ylab;         // [N][B] gathered labels (with act)
+    const float* feat;           // else: the data set, [N][S][in] ...
+    const int32_t* labels;       // ... [N][S]
+    const int32_t* batch_idx;    // ... and the round's sample indices [N][B]
+    int S;
+};
+
+// Row s of worker i and its label; a sample index or label out of range is clamped and reported.
+template <bool NC>
+__device__ __forceinline__ const float* head_row(const HeadRows& r, int i, int s, int B, int in, int C, uint32_t* status, int* y) {
+    if (r.act) {
+        if (y) *y = r.ylab[(size_t)i * B + s];
+        return r.act + ((size_t)i * B + s) * in;
+    }
+    int src = load_g<NC>(r.batch_idx + (size_t)i * B + s);
+    if (src < 0 || src >= r.S) {
+        atomicOr(status, DBW_STATUS_BAD_INDEX);
+        src = src < 0 ? 0 : r.S - 1;
+    }
+    if (y) {
+        int lab = __ldg(r.labels + (size_t)i * r.S + src);
+        if (lab < 0 || lab >= C) {
+            atomicOr(status, DBW_STATUS_BAD_INDEX);
+            lab = lab < 0 ? 0 : C - 1;
+        }
+        *y = lab;
+    }
+    return r.feat + ((size_t)i * r.S + src) * in;
+}
+
+// Sample s of worker i by one warp: z = W a + b, dZ = (softmax(z) - onehot(y)) / B, the sample's loss
+// logsumexp(z) - z_y into loss_s[i][s].  CP = compile-time bound on the classes (16 or 32); in is a multiple of 4.
+// A lane adds its features in ascending order, the lanes are then added by a butterfly.
+template <int CP, bool NC>
+__device__ __forceinline__ void head_forward_sample(int i, int s, int B, int in, int C, const HeadRows& rows, const float* W,
+                                                    const float* bias, float* dz, float* loss_s, uint32_t* status) {
+    const int lane = threadIdx.x & 31;
+    int y;
+    const float4* arow = reinterpret_cast<const float4*>(head_row<NC>(rows, i, s, B, in, C, status, &y));
+    const float4* w4 = reinterpret_cast<const float4*>(W);
+    const int in4 = in >> 2;
+    float acc[CP];
+#pragma unroll
+    for (int c = 0; c < CP; ++c) acc[c] = 0.f;
+    for (int k0 = lane; k0 < in4; k0 += 64) {  // two float4 per lane and pass: twice the loads in flight
+        const int k1 = k0 + 32;
+        const bool two = k1 < in4;
+        const float4 a0 = arow[k0];
+        const float4 a1 = two ? arow[k1] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c0 = 0; c0 < CP; c0 += 8) {  // eight classes at a time: sixteen weight loads in flight per lane
+            if (c0 >= C) break;
+            float4 w0[8], w1[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u;
+                w0[u] = c < C ? load_g<NC>(w4 + (size_t)c * in4 + k0) : make_float4(0.f, 0.f, 0.f, 0.f);
+                w1[u] = (c < C && two) ? load_g<NC>(w4 + (size_t)c * in4 + k1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float t = acc[c0 + u];
+                t = fmaf(a0.x, w0[u].x, t); t = fmaf(a0.y, w0[u].y, t); t = fmaf(a0.z, w0[u].z, t); t = fmaf(a0.w, w0[u].w, t);
+                t = fmaf(a1.x, w1[u].x, t); t = fmaf(a1.y, w1[u].y, t); t = fmaf(a1.z, w1[u].z, t); t = fmaf(a1.w, w1[u].w, t);
+                acc[c0 + u] = t;
+            }
+        }
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+        if (c < C) {
+            acc[c] = warp_sum_f(acc[c]) + load_g<NC>(bias + c);
+            mx = fmaxf(mx, acc[c]);
+        }
+    }
+    float sum = 0.f, zy = 0.f;
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+        if (c < C) {
+            if (c == y) zy = acc[c];
+            acc[c] = expf(acc[c] - mx);
+            sum += acc[c];
+        }
+    }
+    const float inv = 1.0f / sum, invB = 1.0f / (float)B;
+    float mine = 0.f;
+#pragma unroll
+    for (int c = 0; c < CP; ++c)
+        if (c < C && c == lane) mine = (acc[c] * inv - (c == y ? 1.f : 0.f)) * invB;
+    if (lane < C) dz[((size_t)i * B + s) * C + lane] = mine;
+    if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+}
+
+// Backward of the last layer for worker i, features [4 k_lo, 4 k_hi) (at most kHeadChunk4 groups of four) by a
+// block of 256 threads.  A warp owns four feature groups; its lanes split the samples eight ways (lane mod 8):
+//   dW[c][f] = sum_s dZ[s][c] a[s][f]: each lane adds its samples in ascending order, a butterfly adds the lanes;
+//   with dz_prev also dZ of the layer before, (sum_c dZ[s][c] W[c][f]) [a[s][f] > 0], classes in ascending order.
+// The block that owns the first features also adds the bias gradient and the worker's mean loss, in sample
+// order.  smem: B * C floats + B 64-bit offsets.  Ends with a block barrier (shared memory free again).
+constexpr int kHeadChunk4 = 32;
+template <int CP, bool NC>
+__device__ __forceinline__ void head_backward_part(int i, int k_lo, int k_hi, int B, int in, int C, const HeadRows& rows,
+                                                   const float* dz, const float* loss_s, const float* W, float* Gw, float* Gb,
+                                                   float* loss, float* dz_prev, float* smem, uint32_t* status) {
+    float* dzs = smem;
+    long long* rowoff = reinterpret_cast<long long*>(smem + ((B * C + 1) & ~1));
+    for (int e = threadIdx.x; e < B * C; e += blockDim.x) dzs[e] = dz[(size_t)i * B * C + e];
+    const float* base = rows.act ? rows.act : rows.feat;
+    for (int s = threadIdx.x; s < B; s += blockDim.x) rowoff[s] = head_row<NC>(rows, i, s, B, in, C, status, nullptr) - base;
+    __syncthreads();
+    if (k_lo == 0) {
+        if ((int)threadIdx.x < C) {
+            float t = 0.f;
+            for (int s = 0; s < B; ++s) t += dzs[s * C + threadIdx.x];
+            Gb[threadIdx.x] = t;
+        }
+        if (threadIdx.x == 32 && loss) {
+            float t = 0.f;
+            for (int s = 0; s < B; ++s) t += loss_s[(size_t)i * B + s];
+            loss[i] = t * (1.0f / (float)B);
+        }
+    }
+    const int lane = threadIdx.x & 31, slice = lane & 7;
+    const int k = k_lo + (int)(threadIdx.x >> 5) * 4 + (lane >> 3);
+    if (k < k_hi) {  // the eight lanes of a feature group stay together
+        float4 acc[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int s = slice; s < B; s += 8) {
+            const float4 a = *(reinterpret_cast<const float4*>(base + rowoff[s]) + k);
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                if (c < C) {
+                    const float d = dzs[s * C + c];
+                    acc[c].x = fmaf(d, a.x, acc[c].x); acc[c].y = fmaf(d, a.y, acc[c].y);
+                    acc[c].z = fmaf(d, a.z, acc[c].z); acc[c].w = fmaf(d, a.w, acc[c].w);
+                }
+            }
+        }
+        const unsigned grp = 0xffu << (lane & 24);
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+            if (c < C) {
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) {
+                    acc[c].x += __shfl_xor_sync(grp, acc[c].x, o); acc[c].y += __shfl_xor_sync(grp, acc[c].y, o);
+                    acc[c].z += __shfl_xor_sync(grp, acc[c].z, o); acc[c].w += __shfl_xor_sync(grp, acc[c].w, o);
+                }
+                if ((c & 7) == slice) reinterpret_cast<float4*>(Gw + (size_t)c * in)[k] = acc[c];
+            }
+        }
+        if (dz_prev) {
+#pragma unroll
+            for (int c = 0; c < CP; ++c)
+                if (c < C) acc[c] = load_g<NC>(reinterpret_cast<const float4*>(W + (size_t)c * in) + k);
+#pragma unroll 4
+            for (int s = slice; s < B; s += 8) {
+                const float4 a = *(reinterpret_cast<const float4*>(base + rowoff[s]) + k);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < CP; ++c) {
+                    if (c < C) {
+                        const float d = dzs[s * C + c];
+                        v.x = fmaf(d, acc[c].x, v.x); v.y = fmaf(d, acc[c].y, v.y);
+                        v.z = fmaf(d, acc[c].z, v.z); v.w = fmaf(d, acc[c].w, v.w);
+                    }
+                }
+                v.x = a.x > 0.f ? v.x : 0.f; v.y = a.y > 0.f ? v.y : 0.f;
+                v.z = a.z > 0.f ? v.z : 0.f; v.w = a.w > 0.f ? v.w : 0.f;
+                reinterpret_cast<float4*>(dz_prev + ((size_t)i * B + s) * in)[k] = v;
+            }
+        }
+    }
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------ selection, weights, times
 // Arrival time used for ordering: NaN sorts last (as +inf) and is reported in the status word.
 __device__ __forceinline__ double order_time(double t, uint32_t* status) {

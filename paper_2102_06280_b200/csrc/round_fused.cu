@@ -69,6 +69,7 @@ struct FusedArgs {
     const float* lr_pw;
     float* loss;
     signed char fwd_var[DBW_MAX_LAYERS], dw_var[DBW_MAX_LAYERS], da_var[DBW_MAX_LAYERS];
+    int head;  // the last layer takes the small-output steps (at most 32 classes)
 };
 
 template <int R, int TK>
@@ -102,7 +103,29 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(Fus
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.B, N = a.N, L = a.L;
 
-    // ---- mini-batch gather; the last block does the selection, the weights and the times instead ----
+    // Last layer of at most 32 classes: forward + loss by a warp per sample, backward by a block per worker and
+    // 128 features, instead of three GEMMs and the loss step.
+    const int Lg = a.head ? L - 1 : L;  // layers that run as GEMMs
+    HeadRows rows{};
+    if (L > 1) {
+        rows.act = a.act[L - 1]; rows.ylab = a.ylab;
+    } else {
+        rows.feat = a.feat; rows.labels = a.labels; rows.batch_idx = a.batch_idx; rows.S = a.S;
+    }
+    float* loss_s = a.act[L];
+    auto head_forward = [&](int first, int step) {
+        for (int item = first * (kThreads / 32) + warp; item < N * B; item += step * (kThreads / 32)) {
+            const int i = item / B;
+            const float* Xi = a.X + (size_t)i * a.ld;
+            if (a.C <= 16)
+                head_forward_sample<16, false>(i, item % B, B, a.dims[L - 1], a.C, rows, Xi + a.w_off[L - 1], Xi + a.b_off[L - 1], a.dz[L], loss_s, a.status);
+            else
+                head_forward_sample<32, false>(i, item % B, B, a.dims[L - 1], a.C, rows, Xi + a.w_off[L - 1], Xi + a.b_off[L - 1], a.dz[L], loss_s, a.status);
+        }
+    };
+
+    // ---- mini-batch gather (a one-layer model with the small-output last layer: its forward pass and loss
+    //      straight from the data set); the last block does the selection, the weights and the times instead ----
     if (blockIdx.x == gridDim.x - 1) {
         for (int i = warp; i < N; i += kThreads / 32)
             select_worker(i, lane, a.rowptr, a.col, a.t, a.t_edge, a.b, a.kept, a.T_nbr_ws, a.waited, a.status, a.plan, 1, a.uniform);
@@ -116,14 +139,16 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(Fus
             for (int k = 1; k < kThreads / 32; ++k) tr = fmax(tr, red[k]);
             if (a.T_round) *a.T_round = tr;
         }
-    } else {  // the grid has at least two blocks
+    } else if (Lg > 0 || !a.head) {  // the grid has at least two blocks
         for (int item = blockIdx.x; item < N * B; item += gridDim.x - 1)
             gather_row(item % B, item / B, B, a.S, a.dims[0], a.C, a.feat, a.labels, a.batch_idx, a.act[0], a.ylab, a.status);
+    } else {
+        head_forward(blockIdx.x, gridDim.x - 1);
     }
     grid.sync();
 
     // ---- forward: Z_l = A_{l-1} W_l^T + b_l, A_l = ReLU(Z_l), logits for the last layer ----
-    for (int l = 0; l < L; ++l) {
+    for (int l = 0; l < Lg; ++l) {
         const int in = a.dims[l], out = a.dims[l + 1];
         GemmArgs g{};
         g.A = a.act[l]; g.sAz = (long long)B * in; g.sAm = in; g.sAk = 1;
@@ -135,15 +160,39 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(Fus
         grid.sync();
     }
 
-    // ---- loss, dZ_L, last layer's bias gradient ----
-    for (int i = blockIdx.x; i < N; i += gridDim.x) {
-        softmax_ce_worker(i, B, a.C, a.act[L], a.ylab, a.dz[L], a.loss, a.G, a.ld, a.b_off[L - 1], sl);
-        __syncthreads();
+    if (a.head) {
+        if (Lg > 0) {
+            head_forward(blockIdx.x, gridDim.x);
+            grid.sync();
+        }
+        // ---- last layer backward: dW_L, db_L, the loss, dZ_{L-1} ----
+        const int in = a.dims[L - 1], in4 = in >> 2;
+        const int chunks = (in4 + kHeadChunk4 - 1) / kHeadChunk4;
+        for (int item = blockIdx.x; item < N * chunks; item += gridDim.x) {
+            const int i = item / chunks, k_lo = (item % chunks) * kHeadChunk4;
+            const int k_hi = min(in4, k_lo + kHeadChunk4);
+            const float* Xi = a.X + (size_t)i * a.ld;
+            float* Gi = a.G + (size_t)i * a.ld;
+            float* dz_prev = L > 1 ? a.dz[L - 1] : nullptr;
+            if (a.C <= 16)
+                head_backward_part<16, false>(i, k_lo, k_hi, B, in, a.C, rows, a.dz[L], loss_s, Xi + a.w_off[L - 1], Gi + a.w_off[L - 1],
+                                              Gi + a.b_off[L - 1], a.loss, dz_prev, smem, a.status);
+            else
+                head_backward_part<32, false>(i, k_lo, k_hi, B, in, a.C, rows, a.dz[L], loss_s, Xi + a.w_off[L - 1], Gi + a.w_off[L - 1],
+                                              Gi + a.b_off[L - 1], a.loss, dz_prev, smem, a.status);
+        }
+        grid.sync();
+    } else {
+        // ---- loss, dZ_L, last layer's bias gradient ----
+        for (int i = blockIdx.x; i < N; i += gridDim.x) {
+            softmax_ce_worker(i, B, a.C, a.act[L], a.ylab, a.dz[L], a.loss, a.G, a.ld, a.b_off[L - 1], sl);
+            __syncthreads();
+        }
+        grid.sync();
     }
-    grid.sync();
 
     // ---- backward ----
-    for (int l = L - 1; l >= 0; --l) {
+    for (int l = Lg - 1; l >= 0; --l) {
         const int in = a.dims[l], out = a.dims[l + 1];
         GemmArgs g{};  // dW_l[o][k] = sum_m dZ[m][o] A_l[m][k]
         g.A = a.dz[l + 1]; g.sAz = (long long)B * out; g.sAm = 1; g.sAk = out;
@@ -258,6 +307,7 @@ int launch_round_fused(dbw_handle* h, const float* X, const double* t, const int
     a.uniform = (h->flags & DBW_WEIGHT_UNIFORM) ? 1 : 0;
     a.mix_then_correct = (h->flags & DBW_ORDER_MIX_THEN_CORRECT) ? 1 : 0;
     a.lr = lr; a.lr_pw = lr_pw; a.loss = loss;
+    a.head = (fp32_head_usable(h) && (((uintptr_t)X | (uintptr_t)h->d_G) & 15) == 0) ? 1 : 0;
     // grid: as many blocks as the widest step has work items, at most one per SM
     const int B = m.batch, N = h->N;
     long long widest = (long long)N * B;  // gather rows
@@ -266,6 +316,8 @@ int launch_round_fused(dbw_handle* h, const float* X, const double* t, const int
         widest = std::max(widest, (long long)((m.dims[l + 1] + 31) / 32) * ((m.dims[l] + 31) / 32) * N);
     }
     widest = std::max<long long>(widest, (h->ld + 4 * kMixGS - 1) / (4 * kMixGS));
+    widest = std::max<long long>(widest, ((long long)N * B + kThreads / 32 - 1) / (kThreads / 32));  // last layer: a warp per sample
+    widest = std::max<long long>(widest, (long long)N * (((m.dims[m.n_layers - 1] >> 2) + kHeadChunk4 - 1) / kHeadChunk4));
     const int grid = (int)std::min<long long>(h->fused->max_blocks, std::max<long long>(widest + 1, 2));
     for (int l = 0; l < m.n_layers; ++l) {
         a.fwd_var[l] = (signed char)pick_variant(B, m.dims[l + 1], m.dims[l], N, grid);
