@@ -269,19 +269,36 @@ def mlp_loss(x, layers, feats, labels):
     return float(np.mean(lse - a[np.arange(len(labels)), np.asarray(labels)]))
 
 
-def mlp_grad(x, layers, feats, labels):
-    """(g, loss): g = mean over the batch of grad f(x; sample) in the layout of x (Eq. 2)."""
+def mlp_grad(x, layers, feats, labels, relu_on=None, margins=None):
+    """(g, loss): g = mean over the batch of grad f(x; sample) in the layout of x (Eq. 2).
+
+    At a pre-activation of exactly zero ReLU has the sub-differential [0, 1]; this function takes 0 there.
+    A finite-precision implementation may see a pre-activation that is zero up to rounding on either side,
+    and both choices are then valid.  `relu_on` maps (layer, sample, unit) (layer = 1 .. L-1, the index of
+    the activation) to True / False and forces that unit on (a = z, derivative 1) or off (a = 0, derivative
+    0); tests use it to compare at a pre-activation closer to zero than fp32 accumulation resolves.
+    `margins`, if a list, receives per hidden layer the array |z| / (|a| |W|^T + |b|): how far, relative to
+    the size of its terms, each pre-activation is from the kink."""
     a0 = np.asarray(feats, dtype=np.float64)
     labels = np.asarray(labels)
     B = a0.shape[0]
     params = unpack_layers(x, layers)
     acts = [a0]
-    pre = []
+    on = []
     a = a0
     for l, (W, bias) in enumerate(params):
         z = a @ W.T + bias
-        pre.append(z)
-        a = np.maximum(z, 0.0) if l < len(params) - 1 else z
+        if l < len(params) - 1:
+            if margins is not None:
+                margins.append(np.abs(z) / np.maximum(np.abs(a) @ np.abs(W).T + np.abs(bias), 1e-300))
+            active = z > 0.0                      # ReLU'(0) = 0
+            for (ll, smp, unit), val in (relu_on or {}).items():
+                if ll == l + 1:
+                    active[smp, unit] = bool(val)
+            on.append(active)
+            a = np.where(active, z, 0.0)
+        else:
+            a = z
         acts.append(a)
     logits = acts[-1]
     zmax = logits.max(axis=1, keepdims=True)
@@ -298,7 +315,7 @@ def mlp_grad(x, layers, feats, labels):
         grads[l] = (dz.T @ acts[l], dz.sum(axis=0))
         if l > 0:
             da = dz @ W
-            dz = da * (pre[l - 1] > 0.0)      # ReLU'(0) = 0
+            dz = da * on[l - 1]
     g = np.concatenate([np.concatenate([gw.ravel(), gb]) for gw, gb in grads])
     return g, loss
 

@@ -376,6 +376,7 @@ bias_grad_bf16_kernel(int out_dim, int B, const bf16* __restrict__ dz, long long
 
 // ----------------------------------------------------------------------------- last layer on CUDA cores
 constexpr int kMaxClasses = 32;
+constexpr size_t kHeadStageBytes = 100 * 1024;  // last-layer weights up to this size are staged in shared memory (two CTAs per SM)
 
 // logits = A W^T + b (A bf16 [B][K], W fp32 master [C][K]), then dZ = (softmax - onehot)/B and the
 // per-sample loss.  A warp takes HS samples at once: each lane owns 8 consecutive k of every
@@ -454,6 +455,109 @@ head_forward_kernel(int B, int K, int C, const bf16* __restrict__ A, const float
         if (lane < C) dzL[((size_t)i * B + s) * C + lane] = (e / sum - (lane == y ? 1.f : 0.f)) / (float)B;
         const float zy = __shfl_sync(0xffffffffu, zl, y & 31);
         if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+    }
+}
+
+// The same step with the layer's weights in shared memory.  head_forward_kernel fetches every weight row
+// again for each pair of samples (L1/L2 latency on every class: 8 % of the fp32 rate on the 1024 -> 10 layer);
+// here a CTA of eight warps stages the worker's W (C x K fp32) once and works through a contiguous range of
+// (worker, 8 HS samples) items, restaging only when the worker changes; a warp takes HS samples at once, so a
+// weight row read from shared memory is used for HS samples.  Same arithmetic and order as head_forward_kernel.
+template <int CP, int HS>
+__global__ void __launch_bounds__(256, 2)
+head_forward_staged_kernel(int N, int B, int K, int C, const bf16* __restrict__ A, const float* __restrict__ X, long long ld,
+                           long long w_off, long long b_off, const int32_t* __restrict__ ylab, float* __restrict__ dzL,
+                           float* __restrict__ loss_s) {
+    extern __shared__ float4 sw4[];  // [C][K]
+    const float* sw = reinterpret_cast<const float*>(sw4);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int groups = (B + 8 * HS - 1) / (8 * HS);  // items per worker
+    const int items = N * groups;
+    const int per = (items + gridDim.x - 1) / gridDim.x;
+    const int it0 = blockIdx.x * per, it1 = min(items, it0 + per);
+    int staged = -1;
+    for (int it = it0; it < it1; ++it) {
+        const int i = it / groups, s0 = (it % groups) * 8 * HS + warp * HS;
+        if (i != staged) {  // the same for all threads of the CTA
+            __syncthreads();
+            const float4* src = reinterpret_cast<const float4*>(X + (size_t)i * ld + w_off);
+            for (int e = threadIdx.x; e < C * K / 4; e += 256) sw4[e] = __ldg(src + e);
+            __syncthreads();
+            staged = i;
+        }
+        if (s0 >= B) continue;  // warp-uniform; the CTA barriers above depend on the item only
+        float acc[HS][CP];
+#pragma unroll
+        for (int u = 0; u < HS; ++u)
+#pragma unroll
+            for (int c = 0; c < CP; ++c) acc[u][c] = 0.f;
+        auto load_a = [&](int kc, uint4 (&raw)[HS]) {
+            const int k = kc + lane * 8;
+#pragma unroll
+            for (int u = 0; u < HS; ++u) {
+                raw[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (k < K && s0 + u < B) raw[u] = __ldg(reinterpret_cast<const uint4*>(A + ((size_t)i * B + s0 + u) * K + k));
+            }
+        };
+        uint4 cur[HS], nxt[HS];
+        load_a(0, cur);
+        for (int kc = 0; kc < K; kc += 256) {
+            load_a(kc + 256, nxt);  // next chunk in flight while this one is used (all zero past the end)
+            const int k = kc + lane * 8;
+            if (k < K) {
+                float av[HS][8];
+#pragma unroll
+                for (int u = 0; u < HS; ++u) {
+                    const uint32_t w4[4] = {cur[u].x, cur[u].y, cur[u].z, cur[u].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {  // bf16 -> fp32 is a 16-bit shift
+                        av[u][2 * e] = __uint_as_float(w4[e] << 16);
+                        av[u][2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < CP; ++c) {
+                    if (c < C) {
+                        const float4 w0 = *reinterpret_cast<const float4*>(sw + (size_t)c * K + k);
+                        const float4 w1 = *reinterpret_cast<const float4*>(sw + (size_t)c * K + k + 4);
+                        const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+                        for (int u = 0; u < HS; ++u)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[u][c] = fmaf(av[u][e], wv[e], acc[u][c]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < HS; ++u) cur[u] = nxt[u];
+        }
+#pragma unroll
+        for (int u = 0; u < HS; ++u) {
+            float z_mine = 0.f;  // lane c ends up holding logit c of sample s0 + u
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                if (c < C) {
+                    float v = acc[u][c];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane == c) z_mine = v;
+                }
+            }
+            const int s = s0 + u;
+            if (s >= B) continue;  // warp-uniform
+            const float zl = lane < C ? z_mine + __ldg(X + (size_t)i * ld + b_off + lane) : -INFINITY;
+            float mx = zl;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            const float e = lane < C ? expf(zl - mx) : 0.f;
+            float sum = e;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const int y = ylab[(size_t)i * B + s];
+            if (lane < C) dzL[((size_t)i * B + s) * C + lane] = (e / sum - (lane == y ? 1.f : 0.f)) / (float)B;
+            const float zy = __shfl_sync(0xffffffffu, zl, y & 31);
+            if (lane == 0) loss_s[(size_t)i * B + s] = (mx + logf(sum)) - zy;
+        }
     }
 }
 
@@ -729,6 +833,8 @@ int grad_bf16_alloc(dbw_handle* h) {
         }
     }
     if (!ok) return DBW_ERR_CUDA;
+    DBW_CUDA(cudaFuncSetAttribute(head_forward_staged_kernel<12, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadStageBytes));
+    DBW_CUDA(cudaFuncSetAttribute(head_forward_staged_kernel<16, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadStageBytes));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     DBW_CUDA(cudaFuncSetAttribute(head_backward_kernel<32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -776,12 +882,23 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
     // last layer, loss, and its backward
     const int K = m.dims[L - 1];
     bf16* dzP = L >= 2 ? st->dZ[L - 1] : nullptr;
-    if (C <= 16)
+    const size_t w_bytes = (size_t)C * K * sizeof(float);
+    if (C <= 16 && w_bytes <= kHeadStageBytes && (m.w_off[L - 1] & 3) == 0) {  // weights staged in shared memory
+        const int items = N * ((B + 31) / 32);
+        const int grid = std::min(items, 2 * h->sm_count);
+        if (C <= 12)  // ten classes: a quarter fewer accumulators than with the 16-class instance
+            head_forward_staged_kernel<12, 4><<<grid, 256, w_bytes, s>>>(N, B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1],
+                                                                         st->ylab, st->dzL, st->loss_s);
+        else
+            head_forward_staged_kernel<16, 4><<<grid, 256, w_bytes, s>>>(N, B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], m.b_off[L - 1],
+                                                                         st->ylab, st->dzL, st->loss_s);
+    } else if (C <= 16) {
         head_forward_kernel<16, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
-    else
+    } else {
         head_forward_kernel<32, 2><<<dim3((B + 7) / 8, N), 128, 0, s>>>(B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1],
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
+    }
     DBW_LAUNCHED();
     if (loss) {
         loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);

@@ -38,16 +38,16 @@ __global__ void bias_grad_kernel(int B, int out_dim, const float* __restrict__ d
 }
 
 // The GEMM for operands whose unit-stride dimension allows 128-bit accesses (every layer whose width and
-// batch are multiples of four).  A CTA of WM warps owns a tile of 16 WM x 64 outputs; a warp owns 16 rows x 64
-// columns of it as 8 x 4 per thread (lane / 16 picks the row half, lane mod 16 the columns), so that per
-// k a warp reads 8 + 4 floats through three 128-bit shared-memory loads of which the two row loads are
-// broadcasts: 32 multiply-adds per thread for about four shared-memory wavefronts per warp, where the
+// batch are multiples of four).  A CTA of WM warps owns a tile of 2 RM WM x 64 outputs; a warp owns 2 RM rows x 64
+// columns of it as RM x 4 per thread (RM = 8 or 4; lane / 16 picks the row half, lane mod 16 the columns), so that per
+// k a warp reads RM + 4 floats through 128-bit shared-memory loads of which the row loads are broadcasts:
+// with RM = 8, 32 multiply-adds per thread for about four shared-memory wavefronts per warp, where the
 // 4 x 4 layout of gemm_simt_kernel needs the same four wavefronts for 16.  Global loads and stores are
 // 128-bit along the operand's unit-stride dimension.  Every output element is summed over k in ascending
 // order, exactly as in gemm_simt_kernel: the two give the same bits.
-template <int WM>
+template <int WM, int RM>
 __global__ void __launch_bounds__(32 * WM) gemm_vec_kernel(GemmArgs g) {
-    constexpr int BM = 16 * WM, BN = 64, TK = 16, THREADS = 32 * WM;
+    constexpr int BM = 2 * RM * WM, BN = 64, TK = 16, THREADS = 32 * WM;
     constexpr int PA = BM * TK / 4 / THREADS, PB = BN * TK / 4 / THREADS;  // float4 per thread and k-step
     __shared__ __align__(16) float As[TK][BM + 4];
     __shared__ __align__(16) float Bs[TK][BN + 4];
@@ -55,9 +55,9 @@ __global__ void __launch_bounds__(32 * WM) gemm_vec_kernel(GemmArgs g) {
     const float* __restrict__ A = g.A + (size_t)z * g.sAz;
     const float* __restrict__ B = g.B + (size_t)z * g.sBz;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int mw = warp * 16 + (lane >> 4) * 8, nw = (lane & 15) * 4;
+    const int mw = warp * 2 * RM + (lane >> 4) * RM, nw = (lane & 15) * 4;
     const bool a_k_fast = g.sAk == 1, b_k_fast = g.sBk == 1;
-    float acc[8][4] = {};
+    float acc[RM][4] = {};
     float4 pa[PA], pb[PB];
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     auto fetch = [&](int k0) {
@@ -110,13 +110,16 @@ __global__ void __launch_bounds__(32 * WM) gemm_vec_kernel(GemmArgs g) {
         fetch(k0 + TK);  // all zero past the end
 #pragma unroll
         for (int kk = 0; kk < TK; ++kk) {
-            const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][mw]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][mw + 4]);
+            float av[RM];
+#pragma unroll
+            for (int i = 0; i < RM; i += 4) {
+                const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][mw + i]);
+                av[i] = a4.x; av[i + 1] = a4.y; av[i + 2] = a4.z; av[i + 3] = a4.w;
+            }
             const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][nw]);
-            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
             const float bv[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < RM; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
         }
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(32 * WM) gemm_vec_kernel(GemmArgs g) {
         for (int j = 0; j < 4; ++j) bb[j] = __ldg(bias + n + j);
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < RM; ++i) {
         const int m = m0 + mw + i;
         if (m >= g.M) break;
         float v[4];
@@ -190,12 +193,16 @@ last_layer_backward_kernel(int B, int in, int C, HeadRows rows, const float* __r
 
 int run_gemm(const GemmArgs& g, int batch, int sm_count, cudaStream_t s) {
     if (gemm_vec_ok(g)) {
+        // 8 x 4 outputs per thread where that still gives every SM several warps, else 4 x 4 (twice the warps
+        // for the same tile), on tiles of 64, 32 or 16 rows
         const long long t64 = (long long)((g.N + 63) / 64) * ((g.M + 63) / 64) * batch;
-        if (t64 >= 2LL * sm_count) {
-            gemm_vec_kernel<4><<<dim3((g.N + 63) / 64, (g.M + 63) / 64, batch), 128, 0, s>>>(g);
-        } else {  // 32 x 64 tiles: twice the CTAs
-            gemm_vec_kernel<2><<<dim3((g.N + 63) / 64, (g.M + 31) / 32, batch), 64, 0, s>>>(g);
-        }
+        const long long t32 = (long long)((g.N + 63) / 64) * ((g.M + 31) / 32) * batch;
+        if (t64 >= 2LL * sm_count)
+            gemm_vec_kernel<4, 8><<<dim3((g.N + 63) / 64, (g.M + 63) / 64, batch), 128, 0, s>>>(g);
+        else if (t32 >= sm_count)
+            gemm_vec_kernel<4, 4><<<dim3((g.N + 63) / 64, (g.M + 31) / 32, batch), 128, 0, s>>>(g);
+        else
+            gemm_vec_kernel<2, 4><<<dim3((g.N + 63) / 64, (g.M + 15) / 16, batch), 64, 0, s>>>(g);
         DBW_LAUNCHED();
         return DBW_OK;
     }

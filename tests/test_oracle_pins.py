@@ -352,6 +352,40 @@ def test_mlp_grad_finite_differences(layers):
         assert abs(fd - g[k]) <= 1e-6 * max(1.0, abs(g[k])), (k, fd, g[k])
 
 
+def test_mlp_grad_subgradient_choice_at_the_kink_matches_one_sided_differences():
+    """A hidden unit whose pre-activation is exactly zero for one sample: with the unit forced on the gradient is
+    the right-hand derivative of the loss in that unit's bias, forced off (the default) the left-hand one; the
+    margins report that unit, and only that unit, as sitting on the kink."""
+    rng = np.random.default_rng(3)
+    layers = [3, 4, 3]
+    d = wl.logical_dim(layers)
+    x = rng.standard_normal(d) * 0.8
+    W0 = x[:12].reshape(4, 3)
+    feats = rng.standard_normal((4, 3))
+    feats[2] = [1.0, 0.0, 0.0]
+    W0[1] = [0.5, 0.25, -2.0]
+    x[12 + 1] = -0.5                      # bias of unit 1: z[sample 2][unit 1] = 0.5 - 0.5 = 0 exactly
+    labels = rng.integers(0, 3, size=4)
+    margins = []
+    g_off, loss = orc.mlp_grad(x, layers, feats, labels, margins=margins)
+    g_on, loss_on = orc.mlp_grad(x, layers, feats, labels, relu_on={(1, 2, 1): True})
+    g_off2, _ = orc.mlp_grad(x, layers, feats, labels, relu_on={(1, 2, 1): False})
+    assert loss == loss_on and np.array_equal(g_off, g_off2)
+    assert margins[0][2, 1] == 0.0 and (np.delete(margins[0].ravel(), 2 * 4 + 1) > 1e-3).all()
+    k = 12 + 1                            # d loss / d bias of unit 1
+    h = 1e-7
+    e = np.zeros(d); e[k] = h
+    right = (_independent_loss(x + e, layers, feats, labels) - loss) / h
+    left = (loss - _independent_loss(x - e, layers, feats, labels)) / h
+    assert abs(right - g_on[k]) < 1e-6 and abs(left - g_off[k]) < 1e-6
+    assert abs(g_on[k] - g_off[k]) > 1e-3  # the two choices really differ here
+    # every entry that does not pass through that unit is the same under both choices
+    same = np.ones(d, dtype=bool)
+    same[3:6] = False                     # row 1 of W0
+    same[k] = False
+    assert np.allclose(g_on[same], g_off[same], atol=1e-15)
+
+
 def test_softmax_regression_closed_form():
     rng = np.random.default_rng(1)
     fin, fout, B = 7, 4, 9
