@@ -236,7 +236,7 @@ __device__ __forceinline__ void bias_grad_col(int i, int o, int B, int out_dim, 
 
 
 // ------------------------------------------------------------------ last layer with at most 32 classes (Eq. 2)
-__device__ __forceinline__ float warp_sum_f(float v) {
+__device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
@@ -320,7 +320,7 @@ __device__ __forceinline__ void head_forward_sample(int i, int s, int B, int in,
 #pragma unroll
     for (int c = 0; c < CP; ++c) {
         if (c < C) {
-            acc[c] = warp_sum_f(acc[c]) + load_g<NC>(bias + c);
+            acc[c] = warp_sum(acc[c]) + load_g<NC>(bias + c);
             mx = fmaxf(mx, acc[c]);
         }
     }
@@ -445,11 +445,6 @@ __device__ __forceinline__ int clamped_b(const int32_t* b, int i, int deg, uint3
     return bi;
 }
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 
 __device__ __forceinline__ double warp_max(double v) {
 #pragma unroll
