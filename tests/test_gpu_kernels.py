@@ -328,7 +328,11 @@ def test_update_backups_bit_exact_and_resume(name):
 
 
 @pytest.mark.parametrize("dims,batch,n", [([784, 10], 32, 8), ([20, 13, 7], 5, 3), ([100, 70, 33, 10], 19, 4),
-                                           ([784, 200, 10], 64, 6)])
+                                           ([784, 200, 10], 64, 6),
+                                           ([64, 48, 24], 12, 3),     # 24 classes: the 32-class instance of the last-layer kernels
+                                           ([256, 128], 40, 3),       # one layer of more than 32 classes: GEMM + loss kernel
+                                           ([8, 5, 8, 4], 6, 3),      # last layer's weights not 16-byte aligned in the row: GEMM path
+                                           ([128, 64, 64, 12], 256, 5)])  # whole tiles of the 128-bit GEMM, 8 x 4 outputs per thread
 def test_grad_fp32_matches_oracle(dims, batch, n):
     p = _dbw()
     rowptr, col = wl.ring(max(n, 3)) if n >= 3 else wl.path(n)
