@@ -183,12 +183,12 @@ template <int CP>
 __global__ void __launch_bounds__(256)
 last_layer_backward_kernel(int B, int in, int C, HeadRows rows, const float* __restrict__ dz, const float* __restrict__ loss_s,
                            const float* __restrict__ X, float* __restrict__ G, long long ld, long long w_off, long long b_off,
-                           float* __restrict__ loss, float* __restrict__ dz_prev, uint32_t* status) {
+                           float* __restrict__ loss, float* __restrict__ dz_prev, long long b_off_prev, uint32_t* status) {
     extern __shared__ __align__(16) float head_smem[];
     const int i = blockIdx.y, k_lo = blockIdx.x * kHeadChunk4;
     const int k_hi = min(in >> 2, k_lo + kHeadChunk4);
     head_backward_part<CP, true>(i, k_lo, k_hi, B, in, C, rows, dz, loss_s, X + (size_t)i * ld + w_off, G + (size_t)i * ld + w_off,
-                                 G + (size_t)i * ld + b_off, loss, dz_prev, head_smem, status);
+                                 G + (size_t)i * ld + b_off, loss, dz_prev, G + (size_t)i * ld + b_off_prev, head_smem, status);
 }
 
 int run_gemm(const GemmArgs& g, int batch, int sm_count, cudaStream_t s) {
@@ -287,13 +287,13 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
                                                                           h->d_dz[L], loss_s, h->d_status);
             DBW_LAUNCHED();
             last_layer_backward_kernel<16><<<bgrid, 256, smem, s>>>(B, in, C, rows, h->d_dz[L], loss_s, X, G, h->ld, m.w_off[L - 1],
-                                                                    m.b_off[L - 1], loss, dz_prev, h->d_status);
+                                                                    m.b_off[L - 1], loss, dz_prev, L > 1 ? m.b_off[L - 2] : 0, h->d_status);
         } else {
             last_layer_forward_kernel<32><<<(N * B + 7) / 8, 256, 0, s>>>(N, B, in, C, rows, X, h->ld, m.w_off[L - 1], m.b_off[L - 1],
                                                                           h->d_dz[L], loss_s, h->d_status);
             DBW_LAUNCHED();
             last_layer_backward_kernel<32><<<bgrid, 256, smem, s>>>(B, in, C, rows, h->d_dz[L], loss_s, X, G, h->ld, m.w_off[L - 1],
-                                                                    m.b_off[L - 1], loss, dz_prev, h->d_status);
+                                                                    m.b_off[L - 1], loss, dz_prev, L > 1 ? m.b_off[L - 2] : 0, h->d_status);
         }
         DBW_LAUNCHED();
     } else {
@@ -309,7 +309,7 @@ int launch_grad_fp32(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         g.C = G + m.w_off[l]; g.sCz = h->ld; g.sCm = in;
         g.M = out; g.N = in; g.K = B;
         if ((rc = run_gemm(g, N, h->sm_count, s)) != DBW_OK) return rc;
-        if (l < L - 1) {  // the last layer's bias gradient came out of the loss kernel
+        if (l < L - 1 && !(head && l == L - 2)) {  // the last layer's bias gradient came out of the loss kernel, the one before's out of the last layer's backward kernel
             bias_grad_kernel<<<dim3((out + 127) / 128, N), 128, 0, s>>>(B, out, h->d_dz[l + 1], G, h->ld, m.b_off[l]);
             DBW_LAUNCHED();
         }

@@ -345,14 +345,15 @@ __device__ __forceinline__ void head_forward_sample(int i, int s, int B, int in,
 // Backward of the last layer for worker i, features [4 k_lo, 4 k_hi) (at most kHeadChunk4 groups of four) by a
 // block of 256 threads.  A warp owns four feature groups; its lanes split the samples eight ways (lane mod 8):
 //   dW[c][f] = sum_s dZ[s][c] a[s][f]: each lane adds its samples in ascending order, a butterfly adds the lanes;
-//   with dz_prev also dZ of the layer before, (sum_c dZ[s][c] W[c][f]) [a[s][f] > 0], classes in ascending order.
+//   with dz_prev also dZ of the layer before, (sum_c dZ[s][c] W[c][f]) [a[s][f] > 0], classes in ascending order,
+//   and that layer's bias gradient (the sum of its dZ over the samples) into Gb_prev.
 // The block that owns the first features also adds the bias gradient and the worker's mean loss, in sample
 // order.  smem: B * C floats + B 64-bit offsets.  Ends with a block barrier (shared memory free again).
 constexpr int kHeadChunk4 = 32;
 template <int CP, bool NC>
 __device__ __forceinline__ void head_backward_part(int i, int k_lo, int k_hi, int B, int in, int C, const HeadRows& rows,
                                                    const float* dz, const float* loss_s, const float* W, float* Gw, float* Gb,
-                                                   float* loss, float* dz_prev, float* smem, uint32_t* status) {
+                                                   float* loss, float* dz_prev, float* Gb_prev, float* smem, uint32_t* status) {
     float* dzs = smem;
     long long* rowoff = reinterpret_cast<long long*>(smem + ((B * C + 1) & ~1));
     for (int e = threadIdx.x; e < B * C; e += blockDim.x) dzs[e] = dz[(size_t)i * B * C + e];
@@ -405,6 +406,7 @@ __device__ __forceinline__ void head_backward_part(int i, int k_lo, int k_hi, in
 #pragma unroll
             for (int c = 0; c < CP; ++c)
                 if (c < C) acc[c] = load_g<NC>(reinterpret_cast<const float4*>(W + (size_t)c * in) + k);
+            float4 db = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
             for (int s = slice; s < B; s += 8) {
                 const float4 a = *(reinterpret_cast<const float4*>(base + rowoff[s]) + k);
@@ -420,6 +422,16 @@ __device__ __forceinline__ void head_backward_part(int i, int k_lo, int k_hi, in
                 v.x = a.x > 0.f ? v.x : 0.f; v.y = a.y > 0.f ? v.y : 0.f;
                 v.z = a.z > 0.f ? v.z : 0.f; v.w = a.w > 0.f ? v.w : 0.f;
                 reinterpret_cast<float4*>(dz_prev + ((size_t)i * B + s) * in)[k] = v;
+                db.x += v.x; db.y += v.y; db.z += v.z; db.w += v.w;
+            }
+            // bias gradient of the layer before: this lane's samples in ascending order, then the eight lanes
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) {
+                db.x += __shfl_xor_sync(grp, db.x, o); db.y += __shfl_xor_sync(grp, db.y, o);
+                db.z += __shfl_xor_sync(grp, db.z, o); db.w += __shfl_xor_sync(grp, db.w, o);
+            }
+            if (slice == 0) {
+                Gb_prev[4 * k] = db.x; Gb_prev[4 * k + 1] = db.y; Gb_prev[4 * k + 2] = db.z; Gb_prev[4 * k + 3] = db.w;
             }
         }
     }

@@ -176,10 +176,10 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(Fus
             float* dz_prev = L > 1 ? a.dz[L - 1] : nullptr;
             if (a.C <= 16)
                 head_backward_part<16, false>(i, k_lo, k_hi, B, in, a.C, rows, a.dz[L], loss_s, Xi + a.w_off[L - 1], Gi + a.w_off[L - 1],
-                                              Gi + a.b_off[L - 1], a.loss, dz_prev, smem, a.status);
+                                              Gi + a.b_off[L - 1], a.loss, dz_prev, Gi + (L > 1 ? a.b_off[L - 2] : 0), smem, a.status);
             else
                 head_backward_part<32, false>(i, k_lo, k_hi, B, in, a.C, rows, a.dz[L], loss_s, Xi + a.w_off[L - 1], Gi + a.w_off[L - 1],
-                                              Gi + a.b_off[L - 1], a.loss, dz_prev, smem, a.status);
+                                              Gi + a.b_off[L - 1], a.loss, dz_prev, Gi + (L > 1 ? a.b_off[L - 2] : 0), smem, a.status);
         }
         grid.sync();
     } else {
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) round_fused_kernel(Fus
         g.C = a.G + a.w_off[l]; g.sCz = a.ld; g.sCm = in;
         g.M = out; g.N = in; g.K = B;
         gemm_any(a.dw_var[l], g, N, smem);
-        if (l < L - 1)  // the last layer's bias gradient came out of the loss step
+        if (l < L - 1 && !(a.head && l == L - 2))  // the last layer's bias gradient came out of the loss step, the one before's out of the last layer's backward step
             for (int e = blockIdx.x * kThreads + tid; e < N * out; e += gridDim.x * kThreads)
                 bias_grad_col(e / out, e % out, B, out, a.dz[l + 1], a.G, a.ld, a.b_off[l]);
         if (l > 0) {  // dZ_l[m][k] = (sum_o dZ_{l+1}[m][o] W_l[o][k]) * [A_l[m][k] > 0]
