@@ -346,15 +346,12 @@ __global__ void gather_labels_kernel(int B, int S, int C, const int32_t* __restr
 }
 
 // db[o] = sum over the batch of dZ[s][o] (dZ bf16 [B][out], out even).  A block of 256 threads owns 128
-// outputs: a thread sums two adjacent outputs (one 32-bit load per sample) over every fourth sample,
-// and the four partial sums are added through shared memory in a fixed order.
-__global__ void __launch_bounds__(256)
-bias_grad_bf16_kernel(int out_dim, int B, const bf16* __restrict__ dz, long long dz_z, float* __restrict__ G, long long ld,
-                      long long b_off) {
-    __shared__ float2 part[4][64];
-    const int i = blockIdx.y;
+// outputs (block bx of worker i): a thread sums two adjacent outputs (one 32-bit load per sample) over every
+// fourth sample, and the four partial sums are added through shared memory in a fixed order.
+__device__ __forceinline__ void bias_grad_bf16_block(int bx, int i, int out_dim, int B, const bf16* __restrict__ dz, long long dz_z,
+                                                     float* __restrict__ G, long long ld, long long b_off, float2 (*part)[64]) {
     const int pair = threadIdx.x & 63, slice = threadIdx.x >> 6;
-    const int o = blockIdx.x * 128 + 2 * pair;
+    const int o = bx * 128 + 2 * pair;
     float2 s = make_float2(0.f, 0.f);
     if (o < out_dim) {
         const bf16* p = dz + (size_t)i * dz_z + o;
@@ -561,8 +558,10 @@ head_forward_staged_kernel(int N, int B, int K, int C, const bf16* __restrict__ 
     }
 }
 
-__global__ void loss_reduce_kernel(int B, const float* __restrict__ loss_s, float* __restrict__ loss) {
-    const int i = blockIdx.x, lane = threadIdx.x;
+// Mean loss of worker i from its per-sample losses, by the first warp of a block (fixed order).
+__device__ __forceinline__ void loss_reduce_block(int i, int B, const float* __restrict__ loss_s, float* __restrict__ loss) {
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
     float s = 0.f;
     for (int m = lane; m < B; m += 32) s += loss_s[(size_t)i * B + m];
 #pragma unroll
@@ -666,12 +665,11 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
             for (int q = 0; q < KPT; ++q) dst[(size_t)c * K + k + q] = dw[c][q];
 }
 
-// dW of the last layer = sum of the batch parts' partial sums (fixed order), and db[c] = sum_s dZ[s][c].
-__global__ void __launch_bounds__(256)
-head_reduce_kernel(int B, int K, int C, int parts, int workers, const float* __restrict__ dwp, const float* __restrict__ dzL,
-                   float* __restrict__ G, long long ld, long long w_off, long long b_off) {
-    const int i = blockIdx.y;
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+// dW of the last layer = sum of the batch parts' partial sums (fixed order), and db[c] = sum_s dZ[s][c]; block bx of worker i.
+__device__ __forceinline__ void head_reduce_block(int bx, int i, int B, int K, int C, int parts, int workers, const float* __restrict__ dwp,
+                                                  const float* __restrict__ dzL, float* __restrict__ G, long long ld, long long w_off,
+                                                  long long b_off) {
+    const int e = bx * 256 + threadIdx.x;
     if (parts > 1 && e < C * K) {
         float t = 0.f;
         for (int z = 0; z < parts; ++z) t += dwp[((size_t)z * workers + i) * C * K + e];
@@ -682,6 +680,41 @@ head_reduce_kernel(int B, int K, int C, int parts, int workers, const float* __r
         for (int s = 0; s < B; ++s) t += dzL[((size_t)i * B + s) * C + e];
         G[(size_t)i * ld + b_off + e] = t;
     }
+}
+
+// Everything of the gradient that is a reduction over the batch and that only the mix needs, in ONE launch
+// after the last GEMM (four launches of 3-19 us each before): the tensor-core layers' bias gradients, the last
+// layer's dW and db from its batch parts, and the workers' mean losses.  blockIdx.y = worker; blockIdx.x
+// selects the task: [first[t], first[t + 1]) = bias gradient of layer t, then the last layer's reduction,
+// then one block for the loss.
+struct TailArgs {
+    int n_bias;
+    int first[DBW_MAX_LAYERS + 2];
+    int out_dim[DBW_MAX_LAYERS];
+    const bf16* dz[DBW_MAX_LAYERS];
+    long long b_off[DBW_MAX_LAYERS];
+    int B, K, C, parts, workers;
+    const float* dwp;
+    const float* dzL;
+    const float* loss_s;
+    float* loss;  // nullable
+    float* G;
+    long long ld, w_off_last, b_off_last;
+};
+
+__global__ void __launch_bounds__(256) grad_tail_kernel(TailArgs a) {
+    __shared__ float2 part[4][64];
+    const int bx = blockIdx.x, i = blockIdx.y;
+    for (int t = 0; t < a.n_bias; ++t)
+        if (bx >= a.first[t] && bx < a.first[t + 1]) {  // the same for all threads of the block
+            bias_grad_bf16_block(bx - a.first[t], i, a.out_dim[t], a.B, a.dz[t], (long long)a.B * a.out_dim[t], a.G, a.ld, a.b_off[t], part);
+            return;
+        }
+    if (bx < a.first[a.n_bias + 1]) {
+        head_reduce_block(bx - a.first[a.n_bias], i, a.B, a.K, a.C, a.parts, a.workers, a.dwp, a.dzL, a.G, a.ld, a.w_off_last, a.b_off_last);
+        return;
+    }
+    if (a.loss) loss_reduce_block(i, a.B, a.loss_s, a.loss);
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -900,10 +933,6 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
                                                                        m.b_off[L - 1], st->ylab, st->dzL, st->loss_s);
     }
     DBW_LAUNCHED();
-    if (loss) {
-        loss_reduce_kernel<<<N, 32, 0, s>>>(B, st->loss_s, loss);
-        DBW_LAUNCHED();
-    }
     const int parts = B >= 64 ? 4 : 1;
     if (C <= 12)  // ten classes: a quarter fewer multiply-adds than with the 16-class instance
         head_backward_kernel<12, 2><<<dim3((K + 127) / 128, N, parts), 64, (size_t)B * 12 * 4, s>>>(
@@ -915,9 +944,6 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         head_backward_kernel<32, 1><<<dim3((K + 63) / 64, N, parts), 64, (size_t)B * 32 * 4, s>>>(
             B, K, C, st->A[L - 1], X, h->ld, m.w_off[L - 1], st->dzL, G, st->dwp, dzP);
     DBW_LAUNCHED();
-    head_reduce_kernel<<<dim3((std::max(C * K, C) + 255) / 256, N), 256, 0, s>>>(B, K, C, parts, N, st->dwp, st->dzL, G, h->ld,
-                                                                              m.w_off[L - 1], m.b_off[L - 1]);
-    DBW_LAUNCHED();
     // backward through the tensor-core layers
     for (int l = L - 2; l >= 0; --l) {
         const int in = m.dims[l], out = m.dims[l + 1];
@@ -926,8 +952,6 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
         w.outf = G + m.w_off[l]; w.outf_z = h->ld; w.outf_pitch = in;
         w.status = h->d_status;
         if ((rc = run_tc(h, st->dwA[l], st->dwB[l], w, N, s, true, true))) return rc;
-        bias_grad_bf16_kernel<<<dim3((out + 127) / 128, N), 256, 0, s>>>(out, B, st->dZ[l + 1], (long long)B * out, G, h->ld, m.b_off[l]);
-        DBW_LAUNCHED();
         if (l >= 1) {
             TcArgs a{};
             a.M = B; a.N = in; a.K = out; a.epi = EPI_DA;
@@ -937,6 +961,25 @@ int launch_grad_bf16(dbw_handle* h, const float* X, const int32_t* batch_idx, fl
             if ((rc = run_tc(h, st->daA[l], st->daB[l], a, N, s, false, true))) return rc;
         }
     }
+    // the reductions over the batch that only the mix needs: bias gradients, last layer's dW and db, losses
+    TailArgs t{};
+    t.n_bias = L - 1;
+    int next = 0;
+    for (int l = 0; l <= L - 2; ++l) {
+        t.first[l] = next;
+        t.out_dim[l] = m.dims[l + 1];
+        t.dz[l] = st->dZ[l + 1];
+        t.b_off[l] = m.b_off[l];
+        next += (m.dims[l + 1] + 127) / 128;
+    }
+    t.first[L - 1] = next;
+    next += (std::max(C * K, C) + 255) / 256;
+    t.first[L] = next;
+    t.B = B; t.K = K; t.C = C; t.parts = parts; t.workers = N;
+    t.dwp = st->dwp; t.dzL = st->dzL; t.loss_s = st->loss_s; t.loss = loss;
+    t.G = G; t.ld = h->ld; t.w_off_last = m.w_off[L - 1]; t.b_off_last = m.b_off[L - 1];
+    grad_tail_kernel<<<dim3(next + 1, N), 256, 0, s>>>(t);
+    DBW_LAUNCHED();
     return DBW_OK;
 }
 
