@@ -579,7 +579,7 @@ head_backward_kernel(int B, int K, int C, const bf16* __restrict__ A, const floa
                      long long w_off, const float* __restrict__ dzL, float* __restrict__ G, float* __restrict__ dwp,
                      bf16* __restrict__ dzP) {
     // blockIdx.z splits the batch (in chunks of 8 samples) so that enough blocks are in flight; with
-    // more than one part the dW partial sums go to dwp [part][worker][C][K] and head_reduce_kernel
+    // more than one part the dW partial sums go to dwp [part][worker][C][K] and grad_tail_kernel
     // adds them in a fixed order.
     extern __shared__ float4 sdz4[];  // [samples of this part][CP] floats
     float* sdz = reinterpret_cast<float*>(sdz4);
