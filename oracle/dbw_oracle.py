@@ -12,10 +12,10 @@ parameter vector w_i (the paper stores workers as columns of W; this is its
 transpose); deg_i neighbours, b_i backup workers, p_i = deg_i - b_i neighbours
 waited for; t_i the time at which worker i's local update is available.
 
-What each function is pinned by is listed in tests/test_oracle_pins.py.  The
-paper prints no worked numerical round, so absolute per-round values are pinned
-only through invariants, closed forms, brute force and a hand-derived example
-("parity unpinned" by printed values of the paper).
+Every function is pinned by something other than itself; what pins which is
+listed in tests/test_oracle_pins.py: invariants, closed forms, brute force on
+tiny inputs, finite differences and hand-derived examples.  The paper prints no
+worked numerical round, so none of the pins is a value printed by the paper.
 """
 from __future__ import annotations
 
