@@ -9,7 +9,11 @@ round_times      <- hand example; T <= max t, = max t when every p >= 1; = theta
 Dtur             <- hand example; theta is the credited link's establishment time; symmetric masks;
                     each epoch credits every link of P once and its kept links connect the graph
 mlp_grad         <- central finite differences of an independently written loss; softmax-regression
-                    closed form X^T (softmax - Y) / B
+                    closed form X^T (softmax - Y) / B; the sub-gradient choice at a ReLU kink (relu_on) by
+                    one-sided differences, the margins by a unit placed exactly on the kink
+mlp_loss         <- the independently written loss
+spanning_links   <- hand example (the link list of a 4-worker path); N - 1 links that connect the graph (Dtur invariants)
+dbw_round        <- hand example; the network-mean recursion, the consensus limit and the special cases run through it
 """
 import itertools
 import json
