@@ -609,6 +609,10 @@ def summary(res, world, args):
         "terms_per_output": 1.0 + res["kept_last"] / w.N, "bytes_per_launch": operand_bytes, "achieved": operand_rate,
         "peak": smem_peak, "unit": "GB/s", "frac": operand_rate / smem_peak,
         "peak_kind": "128 B/clk/SM x %d SMs x %.0f MHz (shared-memory data pipe, nominal)" % (res["sms"], peaks.get("sm_max_mhz", 1965.0))}
+    if mix_ms <= 0:   # the whole round was one launch (small fp32 networks): there is no mix stage of its own to rate
+        out["roofline"].update({"kernel": "round_fused_kernel", "achieved": None, "frac": None, "frac_of_8TBps_nominal": None,
+                                "note": "one cooperative launch per round; launch-bound, no separate mix kernel"})
+        out["roofline"]["operand_delivery"].update({"achieved": None, "frac": None})
     if res.get("graph_ms"):
         out["cuda_graph"] = {"rounds_per_graph": args.graph, "ms_per_step": res["graph_ms"] / args.steps,
                              "value": aggregate_value(w.N, args.steps, res["graph_ms"], world, sharded),
